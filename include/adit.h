@@ -54,6 +54,7 @@ typedef enum {
 #define ADIT_FLAG_NO_GRAPH 2          /* enqueue kernels one by one instead of replaying a cached launch graph */
 #define ADIT_FLAG_NO_PDL 4            /* no programmatic dependent launch between the loop's kernels */
 #define ADIT_FLAG_MMA_SYNC_ATTENTION 8 /* attention on the legacy mma.sync path instead of tcgen05 (comparison aid) */
+#define ADIT_FLAG_NO_PERSISTENT 16    /* small batches also take the kernel-per-phase path (comparison aid) */
 
 typedef struct adit_handle adit_handle; /* opaque; owns packed weights and a workspace on one device */
 
@@ -173,7 +174,7 @@ int64_t adit_kernel_launches(adit_handle* h);
  * the device, adds up the elapsed milliseconds and launch counts per class into the two arrays of
  * ADIT_N_KERNEL_CLASSES entries, and clears the record.  adit_profile_class_name(i) names class i.
  */
-#define ADIT_N_KERNEL_CLASSES 10
+#define ADIT_N_KERNEL_CLASSES 11
 int adit_profile_enable(adit_handle* h, int on);
 int adit_profile_read(adit_handle* h, double* total_ms, int64_t* launches);
 const char* adit_profile_class_name(int cls);
@@ -192,6 +193,41 @@ const char* adit_profile_class_name(int cls);
  */
 int adit_trace_enable(adit_handle* h, int on);
 int64_t adit_trace_read(adit_handle* h, int64_t* records, int64_t max_records);
+
+/*
+ * adit_clear_status: synchronise the device and reset the status word to ADIT_OK (after an ADIT_E_TIMEOUT has
+ * been read with adit_poll_status; the handle stays usable).
+ */
+int adit_clear_status(adit_handle* h);
+
+/*
+ * adit_uses_persistent_loop: the number of thread blocks the single persistent kernel would use for a call
+ * with B requests and this sm_budget, or 0 when such a call takes the kernel-per-phase path (host only).
+ * Small batches (at most 64 suffix tokens in total, at most 4 requests) of bf16 handles run the whole loop as one
+ * resident kernel of 8-block clusters (section 4.1.1: the stage as one executable on its stream; section 4.1.2: on
+ * its share of the SMs): floor(sm_budget / 8) clusters, at most what the device keeps resident.  Results of the
+ * two paths differ by rounding order only; within a path they do not depend on B, slot or sm_budget.
+ */
+int adit_uses_persistent_loop(adit_handle* h, int B, int sm_budget);
+
+/*
+ * adit_debug_wait_limit: test aid for the bounded device-side waits of the persistent kernel (no counterpart in
+ * the paper).  Sets the limit of every wait to limit_ms milliseconds (default 2000) and, with withhold_level in
+ * 0..7 (embed-in, embed-out, qkv, attention, o, gate/up, down, read-out), makes block 0 withhold its first
+ * completion signal of that level, so that the waits for it run out: the kernel then returns normally,
+ * adit_poll_status reports ADIT_E_TIMEOUT and the call's output is unspecified.  -1 withholds nothing.
+ */
+int adit_debug_wait_limit(adit_handle* h, int limit_ms, int withhold_level);
+
+/*
+ * adit_loop_trace_read: timeline of the most recent persistent-kernel call made while adit_trace_enable was on
+ * (measurement aid).  Per level of the call, in order, seven int64: level type (as in adit_debug_wait_limit),
+ * blocks that took part, earliest and latest time a block saw the level's dependency satisfied, latest time a
+ * block's accumulator (projection) or key loop (attention) was complete, latest time the exchange inside the
+ * clusters was complete, latest time a block had published its part (%globaltimer, ns).  Returns the number of
+ * levels written or a negative status.
+ */
+int64_t adit_loop_trace_read(adit_handle* h, int64_t* records, int64_t max_records);
 
 /* adit_strerror: static string for a status code. */
 const char* adit_strerror(int code);

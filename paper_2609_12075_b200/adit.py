@@ -21,13 +21,14 @@ lib = C.CDLL(_LIB_PATH)
 
 OK, E_INVALID, E_CAPACITY, E_NOT_LOADED, E_UNSUPPORTED, E_CUDA, E_TIMEOUT = 0, -1, -2, -3, -4, -5, -6
 DTYPE_FP32, DTYPE_BF16 = 0, 1
-FLAG_REFERENCE_KERNELS, FLAG_NO_GRAPH, FLAG_NO_PDL, FLAG_MMA_SYNC_ATTENTION = 1, 2, 4, 8
+FLAG_REFERENCE_KERNELS, FLAG_NO_GRAPH, FLAG_NO_PDL, FLAG_MMA_SYNC_ATTENTION, FLAG_NO_PERSISTENT = 1, 2, 4, 8, 16
 MAX_BATCH, MAX_STEPS = 64, 64
 
 EXPORTS = ["adit_create", "adit_load_weights", "adit_denoise", "adit_denoise_host", "adit_destroy",
            "adit_poll_status", "adit_last_cuda_error", "adit_kernel_launches", "adit_strerror",
            "adit_debug_copy", "adit_debug_gemm", "adit_debug_plan", "adit_debug_gemm_stamps", "adit_debug_attention", "adit_attention_static", "adit_profile_enable", "adit_profile_read", "adit_profile_class_name", "adit_trace_enable", "adit_trace_read",
-           "adit_bg_gemm_create", "adit_bg_gemm_launch", "adit_bg_gemm_destroy"]
+           "adit_bg_gemm_create", "adit_bg_gemm_launch", "adit_bg_gemm_destroy",
+           "adit_clear_status", "adit_uses_persistent_loop", "adit_debug_wait_limit", "adit_loop_trace_read"]
 
 
 class Config(C.Structure):
@@ -57,7 +58,7 @@ lib.adit_strerror.argtypes = [C.c_int]
 lib.adit_strerror.restype = C.c_char_p
 lib.adit_debug_copy.argtypes = [C.c_void_p, C.c_char_p, C.c_void_p, C.c_size_t]
 lib.adit_debug_copy.restype = C.c_int64
-N_KERNEL_CLASSES = 10
+N_KERNEL_CLASSES = 11
 lib.adit_debug_gemm_stamps.argtypes = [C.c_void_p, C.c_int]
 lib.adit_debug_plan.argtypes = [C.c_int] * 5 + [C.POINTER(C.c_int32)]
 lib.adit_debug_plan.restype = C.c_int
@@ -74,6 +75,11 @@ STATIC_SCRATCH_BYTES = 8 << 20
 lib.adit_trace_enable.argtypes = [C.c_void_p, C.c_int]
 lib.adit_trace_read.argtypes = [C.c_void_p, C.POINTER(C.c_int64), C.c_int64]
 lib.adit_trace_read.restype = C.c_int64
+lib.adit_clear_status.argtypes = [C.c_void_p]
+lib.adit_uses_persistent_loop.argtypes = [C.c_void_p, C.c_int, C.c_int]
+lib.adit_debug_wait_limit.argtypes = [C.c_void_p, C.c_int, C.c_int]
+lib.adit_loop_trace_read.argtypes = [C.c_void_p, C.POINTER(C.c_int64), C.c_int64]
+lib.adit_loop_trace_read.restype = C.c_int64
 lib.adit_bg_gemm_create.argtypes = [C.c_int, C.c_int, C.c_int, C.c_int, C.POINTER(C.c_void_p)]
 lib.adit_bg_gemm_launch.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_void_p]
 lib.adit_bg_gemm_destroy.argtypes = [C.c_void_p]
@@ -197,6 +203,25 @@ class ADiT:
         release, first/last main loop finished (ns)."""
         buf = np.zeros((max_records, 10), dtype=np.int64)
         n = lib.adit_trace_read(self._h, buf.ctypes.data_as(C.POINTER(C.c_int64)), max_records)
+        if n < 0:
+            raise AditError(int(n))
+        return buf[:n]
+
+    def clear_status(self):
+        self._check(lib.adit_clear_status(self._h))
+
+    def persistent_blocks(self, batch: int, sm_budget: int = 0) -> int:
+        """Thread blocks of the single persistent kernel for such a call, 0 if it takes the kernel-per-phase path."""
+        return int(lib.adit_uses_persistent_loop(self._h, int(batch), int(sm_budget)))
+
+    def debug_wait_limit(self, limit_ms: int, withhold_level: int = -1):
+        self._check(lib.adit_debug_wait_limit(self._h, int(limit_ms), int(withhold_level)))
+
+    def loop_trace_read(self, max_records: int = 8192) -> np.ndarray:
+        """[n_levels, 7] int64 per level of the last traced persistent call: type, blocks, first/last start,
+        last accumulator complete, last exchange complete, last published (ns)."""
+        buf = np.zeros((max_records, 7), dtype=np.int64)
+        n = lib.adit_loop_trace_read(self._h, buf.ctypes.data_as(C.POINTER(C.c_int64)), max_records)
         if n < 0:
             raise AditError(int(n))
         return buf[:n]

@@ -19,6 +19,8 @@
 #include "attention.cuh"
 #include "attention_tc.cuh"
 #include "tc_aux_kernels.cuh"
+#include "loop_kernel.cuh"
+#include <mutex>
 
 using namespace adit;
 
@@ -79,12 +81,24 @@ struct adit_handle {
   bool profiling = false;
   struct ProfRec { int cls; cudaEvent_t a, b; };
   std::vector<ProfRec> prof;
+  // persistent small-batch loop (loop_kernel.cuh)
+  bool loop_ok = false;            // the shape family and the device can run it
+  int loop_clusters = 0;           // clusters of 8 blocks that are resident at once on this device
+  CUtensorMap* maps_dev = 0;       // tensor maps of the loop kernel, device memory
+  uint32_t* loop_counters = 0;     // level counters + abort word
+  loop::GemmLv loop_g[loop::G_COUNT];
+  cudaEvent_t loop_ev = 0;         // end of this handle's most recent persistent call
+  unsigned long long wait_limit_ns = 2000000000ull;  // bound of every device-side wait of the loop kernel
+  int debug_skip_level = -1;       // test aid (adit_debug_wait_limit)
+  unsigned long long* loop_trace = 0;  // [levels][blocks][4] timestamps of the most recent call while tracing
+  size_t loop_trace_cap = 0;
+  int loop_trace_levels = 0, loop_trace_blocks = 0, loop_trace_layers = 0;
 };
 
 // Kernel classes for the optional per-launch device timing (adit_profile_*).
 enum KernelClass : int {
   KC_PROLOGUE = 0, KC_EMBED, KC_NORM, KC_GEMM_QKV, KC_ATTENTION, KC_GEMM_O, KC_GEMM_GATEUP, KC_GEMM_DOWN,
-  KC_FINAL, KC_REDUCE, KC_COUNT
+  KC_FINAL, KC_REDUCE, KC_LOOP, KC_COUNT
 };
 static_assert(KC_COUNT == ADIT_N_KERNEL_CLASSES, "header and library disagree on the class count");
 
@@ -105,6 +119,9 @@ static int dev_alloc(adit_handle* h, void** p, size_t bytes) {
   void* q = nullptr;
   CU_TRY(h, cudaMalloc(&q, bytes < 256 ? 256 : bytes));
   h->allocs.push_back(q);
+  // Padding rows of the activation buffers are read as MMA operands (their results are discarded): they must hold
+  // finite values, never what the allocator left behind.
+  CU_TRY(h, cudaMemset(q, 0, bytes < 256 ? 256 : bytes));
   *p = q;
   return ADIT_OK;
 }
@@ -146,7 +163,12 @@ static AttnPlan plan_attention(const adit_handle* h, int B) {
   return p;
 }
 
+struct LoopInFlight { adit_handle* h; int device; cudaEvent_t ev; int clusters; };
+static std::mutex g_loop_mutex;
+static std::vector<LoopInFlight> g_loop_inflight;
 static cudaError_t init_attention_attrs();
+static int loop_init(adit_handle* h);
+static int loop_build_maps(adit_handle* h);
 static const int ROW_PAD = 320;  // rows beyond the last token that a token tile (<= 256 wide, remapped rows) may touch
 static bool use_reference_kernels(const adit_config& c) {
   return c.dtype == ADIT_DTYPE_FP32 || (c.flags & ADIT_FLAG_REFERENCE_KERNELS);
@@ -241,8 +263,10 @@ extern "C" int adit_create(const adit_config* cfg, int device, adit_handle** out
     if (!h->q_tma) memset(&h->m_q, 0, sizeof(h->m_q));
     if (cudaStreamCreateWithFlags(&h->cap_stream, cudaStreamNonBlocking) != cudaSuccess) return fail(ADIT_E_CUDA);
     if (init_attention_attrs() != cudaSuccess) return fail(ADIT_E_CUDA);
-    h->use_graph = !(c.flags & ADIT_FLAG_NO_GRAPH) && !getenv("ADIT_NO_GRAPH");
-    h->use_pdl = !(c.flags & ADIT_FLAG_NO_PDL) && !getenv("ADIT_NO_PDL");
+    h->use_graph = !(c.flags & ADIT_FLAG_NO_GRAPH);
+    h->use_pdl = !(c.flags & ADIT_FLAG_NO_PDL);
+    int rc_loop = loop_init(h);
+    if (rc_loop) return fail(rc_loop);
   }
 #undef ALLOC
   if (cudaHostAlloc((void**)&h->status_host, sizeof(int), cudaHostAllocMapped) != cudaSuccess)
@@ -257,6 +281,12 @@ extern "C" int adit_destroy(adit_handle* h) {
   if (!h) return ADIT_OK;
   cudaSetDevice(h->device);
   cudaDeviceSynchronize();
+  {
+    std::lock_guard<std::mutex> lock(g_loop_mutex);
+    for (auto it = g_loop_inflight.begin(); it != g_loop_inflight.end();)
+      it = it->h == h ? g_loop_inflight.erase(it) : it + 1;
+  }
+  if (h->loop_ev) cudaEventDestroy(h->loop_ev);
   for (auto& g : h->graphs) cudaGraphExecDestroy(g.second.exec);
   if (h->cap_stream) cudaStreamDestroy(h->cap_stream);
   for (void* p : h->allocs) cudaFree(p);
@@ -369,6 +399,8 @@ static int pack_all(adit_handle* h) {
            tc::make_map_bf16(&L.m_d, L.wd, D, F, tc::TILE_F);
     }
     if (!ok) return ADIT_E_CUDA;
+    int rc_maps = loop_build_maps(h);
+    if (rc_maps) return rc_maps;
   }
   for (auto& kv : h->raw) cudaFree(kv.second);
   h->raw.clear();
@@ -728,6 +760,228 @@ static int enqueue_tc(adit_handle* h, int B, int K, int G, cudaStream_t st) {
   return ADIT_OK;
 }
 
+
+// ---------------------------------------------------------------------------------------------
+// Persistent small-batch loop: plan, tensor maps, launch
+// ---------------------------------------------------------------------------------------------
+
+// Launches of the loop kernel that may still be running, per process: two of them whose clusters do not fit the
+// device together would each hold part of the SMs and wait for the other's missing blocks.  A call that does not
+// fit beside the ones in flight is ordered behind them on the device (an event wait; the host never blocks).
+
+// k-slices per feature tile for one projection: the choice depends on the shape and on the device's cluster
+// capacity only (never on the call's SM budget or batch), so the order of every sum is fixed.
+static loop::GemmLv plan_loop_gemm(int n_feat, int K, bool dual, int epi, int map_a, int ldo, int clusters_dev) {
+  loop::GemmLv g{};
+  g.n_ftiles = n_feat / 128;
+  g.kb_total = K / 64;
+  g.dual = dual ? 1 : 0; g.epi = epi; g.map_a = map_a; g.ldo = ldo;
+  double best = 1e30;
+  for (int ks = 8; ks >= 2; ks >>= 1) {
+    if (g.kb_total % ks) continue;
+    const int nf = loop::CS / ks, units = (g.n_ftiles + nf - 1) / nf, kbn = g.kb_total / ks;
+    const int rounds = (units + clusters_dev - 1) / clusters_dev;
+    const double cost = rounds * (2.0 + 0.035 * kbn * 4 * (dual ? 2 : 1));
+    if (cost < best - 1e-9) { best = cost; g.ks = ks; g.nf = nf; g.units = units; g.kbn = kbn; }
+  }
+  return g;
+}
+
+template <int DH>
+static cudaError_t loop_prepare_dh(int* clusters) {
+  cudaError_t e = cudaFuncSetAttribute(loop::adit_loop_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, loop::SMEM_BYTES);
+  if (e != cudaSuccess) return e;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(loop::CS * 64);
+  cfg.blockDim = dim3(loop::THREADS);
+  cfg.dynamicSmemBytes = loop::SMEM_BYTES;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = loop::CS; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr; cfg.numAttrs = 1;
+  return cudaOccupancyMaxActiveClusters(clusters, loop::adit_loop_kernel<DH>, &cfg);
+}
+
+// Called from adit_create (tensor-core path): decides whether this shape family and device can run the loop kernel.
+static int loop_init(adit_handle* h) {
+  const adit_config& c = h->cfg;
+  h->loop_ok = false;
+  if (c.flags & ADIT_FLAG_NO_PERSISTENT) return ADIT_OK;
+  const int D = c.d_model, F = c.d_ff, Q = c.n_q_heads * c.head_dim, KV = c.n_kv_heads * c.head_dim, QKV = Q + 2 * KV;
+  const int G = c.n_q_heads / c.n_kv_heads;
+  if (D % 128 || F % 128 || QKV % 128 || Q % 128 || (128 % G) || !h->q_tma) return ADIT_OK;
+  if ((D / 64) % 2 || (Q / 64) % 2 || (F / 64) % 2 || D / 128 > 32) return ADIT_OK;
+  if (h->n_tok > loop::TOK) return ADIT_OK;
+  int clusters = 0;
+  cudaError_t e = c.head_dim == 64 ? loop_prepare_dh<64>(&clusters) : c.head_dim == 128 ? loop_prepare_dh<128>(&clusters) : loop_prepare_dh<256>(&clusters);
+  if (e != cudaSuccess || clusters < 1) { cudaGetLastError(); return ADIT_OK; }
+  h->loop_clusters = clusters;
+  h->loop_g[loop::G_W2] = plan_loop_gemm(D, D, false, loop::LEPI_EMBED, loop::MAP_A_EZ, 0, clusters);
+  h->loop_g[loop::G_QKV] = plan_loop_gemm(QKV, D, false, loop::LEPI_STORE, loop::MAP_A_HB, QKV, clusters);
+  h->loop_g[loop::G_O] = plan_loop_gemm(D, Q, false, loop::LEPI_RESID, loop::MAP_A_ATT, 0, clusters);
+  h->loop_g[loop::G_GU] = plan_loop_gemm(F, D, true, loop::LEPI_GEGLU, loop::MAP_A_HB, F, clusters);
+  h->loop_g[loop::G_DOWN] = plan_loop_gemm(D, F, false, loop::LEPI_RESID, loop::MAP_A_MLP, 0, clusters);
+  for (int i = 0; i < loop::G_COUNT; ++i)
+    if (h->loop_g[i].ks == 0) return ADIT_OK;
+  void* p = nullptr;
+  int rc = dev_alloc(h, &p, sizeof(CUtensorMap) * (size_t)(loop::MAP_LAYER0 + 4 * c.n_layers));
+  if (rc) return rc;
+  h->maps_dev = (CUtensorMap*)p;
+  rc = dev_alloc(h, &p, sizeof(uint32_t) * 2 * loop::LV_COUNT);
+  if (rc) return rc;
+  h->loop_counters = (uint32_t*)p;
+  CU_TRY(h, cudaEventCreateWithFlags(&h->loop_ev, cudaEventDisableTiming));
+  h->loop_ok = true;
+  return ADIT_OK;
+}
+
+// Called when the weights have been packed: the loop kernel's tensor maps, in device memory.
+static int loop_build_maps(adit_handle* h) {
+  if (!h->loop_ok) return ADIT_OK;
+  const adit_config& c = h->cfg;
+  const int64_t D = c.d_model, F = c.d_ff, Q = (int64_t)c.n_q_heads * c.head_dim, KV = (int64_t)c.n_kv_heads * c.head_dim;
+  const int64_t Mx = (int64_t)c.max_batch * h->n_tok + ROW_PAD, Max = (int64_t)c.max_batch * c.horizon + ROW_PAD;
+  std::vector<CUtensorMap> m(loop::MAP_LAYER0 + 4 * (size_t)c.n_layers);
+  bool ok = tc::make_map_bf16(&m[loop::MAP_W2], h->W2, D, D, 128) &&
+            tc::make_map_bf16(&m[loop::MAP_A_EZ], h->ez, Max, D, loop::TOK) &&
+            tc::make_map_bf16(&m[loop::MAP_A_HB], h->hb, Mx, D, loop::TOK) &&
+            tc::make_map_bf16(&m[loop::MAP_A_ATT], h->att, Mx, Q, loop::TOK) &&
+            tc::make_map_bf16(&m[loop::MAP_A_MLP], h->mlp, Mx, F, loop::TOK) &&
+            tc::make_map_bf16(&m[loop::MAP_KV2D], h->qkv, Mx, Q + 2 * KV, attn::KEY_BLOCK);
+  m[loop::MAP_Q3D] = h->m_q;
+  for (int l = 0; l < c.n_layers && ok; ++l) {
+    LayerWeights& L = h->layers[l];
+    ok = tc::make_map_bf16(&m[loop::MAP_LAYER0 + 4 * l + 0], L.wqkv, Q + 2 * KV, D, 128) &&
+         tc::make_map_bf16(&m[loop::MAP_LAYER0 + 4 * l + 1], L.wo, D, Q, 128) &&
+         tc::make_map_bf16(&m[loop::MAP_LAYER0 + 4 * l + 2], L.wgu, 2 * F, D, 128) &&
+         tc::make_map_bf16(&m[loop::MAP_LAYER0 + 4 * l + 3], L.wd, D, F, 128);
+  }
+  if (!ok) return ADIT_E_CUDA;
+  CU_TRY(h, cudaMemcpy(h->maps_dev, m.data(), m.size() * sizeof(CUtensorMap), cudaMemcpyHostToDevice));
+  return ADIT_OK;
+}
+
+// One request's prefix cache as a 3-D tensor (channel, row, plane = (layer, K|V, kv head)) whose row extent is the
+// request's prefix length: rows at or beyond it are never read, the copy engine writes zeros for them.
+static bool make_map_prefix(CUtensorMap* m, const void* base, int dh, int plen, int p_cap, int64_t planes) {
+  tc::EncodeTiledFn fn = tc::encode_tiled_fn();
+  if (!fn) return false;
+  cuuint64_t gdim[3] = {(cuuint64_t)dh, (cuuint64_t)(plen > 0 ? plen : 1), (cuuint64_t)planes};
+  cuuint64_t gstride[2] = {(cuuint64_t)dh * 2, (cuuint64_t)p_cap * dh * 2};
+  cuuint32_t box[3] = {64, (cuuint32_t)attn::KEY_BLOCK, 1};
+  cuuint32_t estr[3] = {1, 1, 1};
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), gdim, gstride, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+static int loop_clusters_for(const adit_handle* h, int sm_budget) {
+  const int G = (sm_budget <= 0 || sm_budget >= h->sm_count) ? h->sm_count : sm_budget;
+  int cl = G / loop::CS;
+  return cl > h->loop_clusters ? h->loop_clusters : cl;
+}
+static bool loop_eligible(const adit_handle* h, int B, int sm_budget) {
+  return h->loop_ok && B <= loop::MAXB && B * h->n_tok <= loop::TOK && loop_clusters_for(h, sm_budget) >= 1;
+}
+
+static int denoise_loop(adit_handle* h, int B, const PrefixTable& pt, const float* state, const float* noise, int K,
+                        int sm_budget, cudaStream_t st, float* out) {
+  const adit_config& c = h->cfg;
+  const int D = c.d_model, A = c.action_dim, S = c.state_dim, Ta = c.horizon;
+  const int clusters = loop_clusters_for(h, sm_budget);
+  loop::LoopParams p{};
+  const int64_t planes = (int64_t)c.n_layers * 2 * c.n_kv_heads;
+  for (int b = 0; b < loop::MAXB; ++b) {
+    p.plen[b] = b < B ? pt.len[b] : 0;
+    if (b < B && pt.len[b] > 0) {
+      if (!make_map_prefix(&p.pk[b], pt.kv[b], c.head_dim, pt.len[b], c.max_prefix_len, planes)) return ADIT_E_CUDA;
+    } else {
+      p.pk[b] = h->m_q;  // never used (no prefix block): any valid map
+    }
+  }
+  p.maps = h->maps_dev;
+  for (int i = 0; i < loop::G_COUNT; ++i) p.g[i] = h->loop_g[i];
+  p.L = c.n_layers; p.K = K; p.D = D; p.F = c.d_ff; p.n_q_heads = c.n_q_heads; p.n_kv_heads = c.n_kv_heads;
+  p.n_tok = h->n_tok; p.horizon = Ta; p.A = A; p.B = B; p.M = B * h->n_tok; p.Ma = B * Ta;
+  p.n_clusters = clusters;
+  const int Gq = c.n_q_heads / c.n_kv_heads;
+  p.n_row_tiles = (h->n_tok * Gq + 127) / 128;
+  p.att_units = B * c.n_kv_heads * p.n_row_tiles;
+  p.ssq_ld = c.max_batch * h->n_tok + ROW_PAD;
+  p.n_dtiles = D / 128;
+  p.scale_log2 = 1.4426950408889634f / sqrtf((float)c.head_dim);
+  p.eps = c.rms_eps; p.dt = 1.0f / (float)K;
+  p.x = h->x; p.h = h->h; p.ssq = h->ssq; p.out = out;
+  p.hb = (bf16*)h->hb; p.qkv = (bf16*)h->qkv; p.att = (bf16*)h->att; p.mlp = (bf16*)h->mlp; p.ez = (bf16*)h->ez;
+  p.Wfold = h->Wfold; p.bfold = h->bfold; p.ctime = h->ctime; p.hs = h->hs; p.ssq_state = h->rstd_state;
+  p.Wout = h->Wout; p.bout = h->bout; p.b2 = h->b2; p.hsb = h->hsb;
+  p.counters = h->loop_counters; p.status = h->status_dev;
+  p.timeout_ns = h->wait_limit_ns; p.debug_skip_level = h->debug_skip_level;
+  const int n_levels = K * (3 + 5 * c.n_layers), n_blocks = clusters * loop::CS;
+  p.trace = nullptr;
+  if (h->tracing) {
+    const size_t need = (size_t)n_levels * n_blocks * 4;
+    if (need > h->loop_trace_cap) {
+      void* q = nullptr;
+      CU_TRY(h, cudaMalloc(&q, need * 8));
+      h->allocs.push_back(q);
+      h->loop_trace = (unsigned long long*)q; h->loop_trace_cap = need;
+    }
+    CU_TRY(h, cudaMemsetAsync(h->loop_trace, 0, need * 8, st));
+    p.trace = h->loop_trace;
+    h->loop_trace_levels = n_levels; h->loop_trace_blocks = n_blocks; h->loop_trace_layers = c.n_layers;
+  }
+  {
+    // order this call behind loop kernels of other handles that it would not fit beside
+    std::lock_guard<std::mutex> lock(g_loop_mutex);
+    int busy = 0;
+    for (auto it = g_loop_inflight.begin(); it != g_loop_inflight.end();) {
+      if (it->h != h && it->device == h->device && cudaEventQuery(it->ev) == cudaSuccess) it = g_loop_inflight.erase(it);
+      else { if (it->h != h && it->device == h->device) busy += it->clusters; ++it; }
+    }
+    cudaGetLastError();  // (cudaErrorNotReady from the queries is not an error)
+    if (busy + clusters > h->loop_clusters)
+      for (auto& e : g_loop_inflight)
+        if (e.h != h && e.device == h->device) CU_TRY(h, cudaStreamWaitEvent(st, e.ev, 0));
+  }
+  {
+    ProfScope ps(h, KC_PROLOGUE, st);
+    int blocks = (p.Ma * A + 255) / 256;
+    if (blocks < B) blocks = B;
+    loop::loop_setup_kernel<<<blocks, 256, 0, st>>>(h->loop_counters, noise, state, h->x, p.Ma * A, h->Ws, h->bs, h->hs, h->hsb,
+                                                   h->rstd_state, B, S, D);
+    h->launches++;
+  }
+  {
+    ProfScope ps(h, KC_LOOP, st);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)n_blocks);
+    cfg.blockDim = dim3(loop::THREADS);
+    cfg.dynamicSmemBytes = loop::SMEM_BYTES;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = loop::CS; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = h->use_pdl ? 2 : 1;
+    cudaError_t e = c.head_dim == 64    ? cudaLaunchKernelEx(&cfg, loop::adit_loop_kernel<64>, p)
+                    : c.head_dim == 128 ? cudaLaunchKernelEx(&cfg, loop::adit_loop_kernel<128>, p)
+                                        : cudaLaunchKernelEx(&cfg, loop::adit_loop_kernel<256>, p);
+    CU_TRY(h, e);
+    h->launches++;
+  }
+  {
+    std::lock_guard<std::mutex> lock(g_loop_mutex);
+    CU_TRY(h, cudaEventRecord(h->loop_ev, st));
+    bool found = false;
+    for (auto& e : g_loop_inflight)
+      if (e.h == h) { e.clusters = clusters; found = true; }
+    if (!found) g_loop_inflight.push_back({h, h->device, h->loop_ev, clusters});
+  }
+  return ADIT_OK;
+}
+
 // Tensor-core loop (bf16).  The per-call descriptor goes to the device through a one-block kernel; the
 // rest of the call is one launch of a graph captured once per (B, K, budget) and cached in the handle.
 static int denoise_tc(adit_handle* h, int B, const PrefixTable& pt, const float* state, const float* noise, int K,
@@ -745,6 +999,7 @@ static int denoise_tc(adit_handle* h, int B, const PrefixTable& pt, const float*
                                                               K, D, Tm, EpiArgs{h->ctime, D, nullptr, h->b1, 0});
     h->ctime_steps = K;
   }
+  if (loop_eligible(h, B, sm_budget)) return denoise_loop(h, B, pt, state, noise, K, sm_budget, st, out);
   CallDesc d;
   d.pt = pt; d.state = state; d.noise = noise; d.out = out;
   set_desc_kernel<<<1, 32, 0, st>>>(d, h->desc_dev);
@@ -835,7 +1090,7 @@ extern "C" int adit_denoise_host(adit_handle* h, int B, const void* const* prefi
 
 extern "C" const char* adit_profile_class_name(int cls) {
   static const char* names[KC_COUNT] = {"prologue", "embed", "norm", "gemm_qkv", "attention", "gemm_o",
-                                        "gemm_gateup", "gemm_down", "final", "reduce"};
+                                        "gemm_gateup", "gemm_down", "final", "reduce", "loop"};
   return (cls >= 0 && cls < KC_COUNT) ? names[cls] : "";
 }
 
@@ -904,6 +1159,58 @@ extern "C" int64_t adit_trace_read(adit_handle* h, int64_t* records, int64_t max
     o[6] = w_max ? (int64_t)w_min : 0; o[7] = (int64_t)w_max;
     o[8] = m_max ? (int64_t)m_min : 0; o[9] = (int64_t)m_max;
     ++n;
+  }
+  return n;
+}
+
+
+extern "C" int adit_clear_status(adit_handle* h) {
+  if (!h) return ADIT_E_INVALID;
+  CU_TRY(h, cudaSetDevice(h->device));
+  CU_TRY(h, cudaDeviceSynchronize());
+  *h->status_host = 0;
+  return ADIT_OK;
+}
+
+extern "C" int adit_debug_wait_limit(adit_handle* h, int limit_ms, int withhold_level) {
+  if (!h || limit_ms < 1 || withhold_level < -1 || withhold_level >= loop::LV_COUNT) return ADIT_E_INVALID;
+  h->wait_limit_ns = (unsigned long long)limit_ms * 1000000ull;
+  h->debug_skip_level = withhold_level;
+  return ADIT_OK;
+}
+
+extern "C" int adit_uses_persistent_loop(adit_handle* h, int B, int sm_budget) {
+  if (!h || B < 1) return ADIT_E_INVALID;
+  if (h->cfg.dtype != ADIT_DTYPE_BF16 || use_reference_kernels(h->cfg)) return 0;
+  return loop_eligible(h, B, sm_budget) ? loop_clusters_for(h, sm_budget) * loop::CS : 0;
+}
+
+extern "C" int64_t adit_loop_trace_read(adit_handle* h, int64_t* records, int64_t max_records) {
+  if (!h || !records || max_records < 0) return ADIT_E_INVALID;
+  if (!h->loop_trace || !h->loop_trace_levels) return 0;
+  CU_TRY(h, cudaSetDevice(h->device));
+  CU_TRY(h, cudaDeviceSynchronize());
+  const int nl = h->loop_trace_levels, nb = h->loop_trace_blocks, per_step = 3 + 5 * h->loop_trace_layers;
+  std::vector<unsigned long long> buf((size_t)nl * nb * 4);
+  CU_TRY(h, cudaMemcpy(buf.data(), h->loop_trace, buf.size() * 8, cudaMemcpyDeviceToHost));
+  int64_t n = 0;
+  for (int lv = 0; lv < nl && n < max_records; ++lv, ++n) {
+    const int j = lv % per_step;
+    const int type = j == 0 ? loop::LV_EMBED_IN : j == 1 ? loop::LV_W2 : j == per_step - 1 ? loop::LV_FINAL : loop::LV_QKV + (j - 2) % 5;
+    unsigned long long s_min = ~0ull, s_max = 0, a_max = 0, x_max = 0, e_max = 0;
+    int blocks = 0;
+    for (int b = 0; b < nb; ++b) {
+      const unsigned long long* t = &buf[((size_t)lv * nb + b) * 4];
+      if (!t[0]) continue;
+      ++blocks;
+      if (t[0] < s_min) s_min = t[0];
+      if (t[0] > s_max) s_max = t[0];
+      if (t[1] > a_max) a_max = t[1];
+      if (t[2] > x_max) x_max = t[2];
+      if (t[3] > e_max) e_max = t[3];
+    }
+    int64_t* o = records + n * 7;
+    o[0] = type; o[1] = blocks; o[2] = blocks ? (int64_t)s_min : 0; o[3] = (int64_t)s_max; o[4] = (int64_t)a_max; o[5] = (int64_t)x_max; o[6] = (int64_t)e_max;
   }
   return n;
 }
