@@ -54,7 +54,7 @@ typedef enum {
 #define ADIT_FLAG_NO_GRAPH 2          /* enqueue kernels one by one instead of replaying a cached launch graph */
 #define ADIT_FLAG_NO_PDL 4            /* no programmatic dependent launch between the loop's kernels */
 #define ADIT_FLAG_MMA_SYNC_ATTENTION 8 /* attention on the legacy mma.sync path instead of tcgen05 (comparison aid) */
-#define ADIT_FLAG_NO_PERSISTENT 16    /* small batches also take the kernel-per-phase path (comparison aid) */
+#define ADIT_FLAG_PERSISTENT_LOOP 16  /* small batches run as one persistent kernel instead of a kernel per phase (see adit_uses_persistent_loop) */
 
 typedef struct adit_handle adit_handle; /* opaque; owns packed weights and a workspace on one device */
 
@@ -221,11 +221,12 @@ int adit_debug_wait_limit(adit_handle* h, int limit_ms, int withhold_level);
 
 /*
  * adit_loop_trace_read: timeline of the most recent persistent-kernel call made while adit_trace_enable was on
- * (measurement aid).  Per level of the call, in order, seven int64: level type (as in adit_debug_wait_limit),
- * blocks that took part, earliest and latest time a block saw the level's dependency satisfied, latest time a
- * block's accumulator (projection) or key loop (attention) was complete, latest time the exchange inside the
- * clusters was complete, latest time a block had published its part (%globaltimer, ns).  Returns the number of
- * levels written or a negative status.
+ * (measurement aid).  Per level of the call, in order, eleven int64: level type (as in adit_debug_wait_limit),
+ * blocks that took part, the earliest time a block saw the level's dependency satisfied, and the latest time over
+ * the blocks of eight events (%globaltimer, ns; 0 where not recorded): dependency seen; accumulator complete
+ * (projection) or key loop complete (attention); partial sums sent; partial sums received; epilogue stored;
+ * level's flag published; first activation tile landed; last product issued.
+ * Returns the number of levels written or a negative status.
  */
 int64_t adit_loop_trace_read(adit_handle* h, int64_t* records, int64_t max_records);
 

@@ -21,7 +21,7 @@ lib = C.CDLL(_LIB_PATH)
 
 OK, E_INVALID, E_CAPACITY, E_NOT_LOADED, E_UNSUPPORTED, E_CUDA, E_TIMEOUT = 0, -1, -2, -3, -4, -5, -6
 DTYPE_FP32, DTYPE_BF16 = 0, 1
-FLAG_REFERENCE_KERNELS, FLAG_NO_GRAPH, FLAG_NO_PDL, FLAG_MMA_SYNC_ATTENTION, FLAG_NO_PERSISTENT = 1, 2, 4, 8, 16
+FLAG_REFERENCE_KERNELS, FLAG_NO_GRAPH, FLAG_NO_PDL, FLAG_MMA_SYNC_ATTENTION, FLAG_PERSISTENT_LOOP = 1, 2, 4, 8, 16
 MAX_BATCH, MAX_STEPS = 64, 64
 
 EXPORTS = ["adit_create", "adit_load_weights", "adit_denoise", "adit_denoise_host", "adit_destroy",
@@ -218,9 +218,10 @@ class ADiT:
         self._check(lib.adit_debug_wait_limit(self._h, int(limit_ms), int(withhold_level)))
 
     def loop_trace_read(self, max_records: int = 8192) -> np.ndarray:
-        """[n_levels, 7] int64 per level of the last traced persistent call: type, blocks, first/last start,
-        last accumulator complete, last exchange complete, last published (ns)."""
-        buf = np.zeros((max_records, 7), dtype=np.int64)
+        """[n_levels, 11] int64 per level of the last traced persistent call: type, blocks, earliest start, then
+        the latest over blocks of: start, accumulator complete, partials sent, partials received, epilogue stored,
+        published, first activation tile landed, last product issued (ns)."""
+        buf = np.zeros((max_records, 11), dtype=np.int64)
         n = lib.adit_loop_trace_read(self._h, buf.ctypes.data_as(C.POINTER(C.c_int64)), max_records)
         if n < 0:
             raise AditError(int(n))

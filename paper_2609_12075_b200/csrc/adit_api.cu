@@ -86,6 +86,7 @@ struct adit_handle {
   int loop_clusters = 0;           // clusters of 8 blocks that are resident at once on this device
   CUtensorMap* maps_dev = 0;       // tensor maps of the loop kernel, device memory
   uint32_t* loop_counters = 0;     // level counters + abort word
+  uint8_t* loop_scratch = 0;       // per-cluster partial sums of the loop kernel
   loop::GemmLv loop_g[loop::G_COUNT];
   cudaEvent_t loop_ev = 0;         // end of this handle's most recent persistent call
   unsigned long long wait_limit_ns = 2000000000ull;  // bound of every device-side wait of the loop kernel
@@ -806,7 +807,7 @@ static cudaError_t loop_prepare_dh(int* clusters) {
 static int loop_init(adit_handle* h) {
   const adit_config& c = h->cfg;
   h->loop_ok = false;
-  if (c.flags & ADIT_FLAG_NO_PERSISTENT) return ADIT_OK;
+  if (!(c.flags & ADIT_FLAG_PERSISTENT_LOOP)) return ADIT_OK;
   const int D = c.d_model, F = c.d_ff, Q = c.n_q_heads * c.head_dim, KV = c.n_kv_heads * c.head_dim, QKV = Q + 2 * KV;
   const int G = c.n_q_heads / c.n_kv_heads;
   if (D % 128 || F % 128 || QKV % 128 || Q % 128 || (128 % G) || !h->q_tma) return ADIT_OK;
@@ -830,6 +831,9 @@ static int loop_init(adit_handle* h) {
   rc = dev_alloc(h, &p, sizeof(uint32_t) * 2 * loop::LV_COUNT);
   if (rc) return rc;
   h->loop_counters = (uint32_t*)p;
+  rc = dev_alloc(h, &p, (size_t)clusters * loop::XS_CLUSTER_BYTES);
+  if (rc) return rc;
+  h->loop_scratch = (uint8_t*)p;
   CU_TRY(h, cudaEventCreateWithFlags(&h->loop_ev, cudaEventDisableTiming));
   h->loop_ok = true;
   return ADIT_OK;
@@ -915,12 +919,12 @@ static int denoise_loop(adit_handle* h, int B, const PrefixTable& pt, const floa
   p.hb = (bf16*)h->hb; p.qkv = (bf16*)h->qkv; p.att = (bf16*)h->att; p.mlp = (bf16*)h->mlp; p.ez = (bf16*)h->ez;
   p.Wfold = h->Wfold; p.bfold = h->bfold; p.ctime = h->ctime; p.hs = h->hs; p.ssq_state = h->rstd_state;
   p.Wout = h->Wout; p.bout = h->bout; p.b2 = h->b2; p.hsb = h->hsb;
-  p.counters = h->loop_counters; p.status = h->status_dev;
+  p.counters = h->loop_counters; p.status = h->status_dev; p.xscratch = h->loop_scratch;
   p.timeout_ns = h->wait_limit_ns; p.debug_skip_level = h->debug_skip_level;
   const int n_levels = K * (3 + 5 * c.n_layers), n_blocks = clusters * loop::CS;
   p.trace = nullptr;
   if (h->tracing) {
-    const size_t need = (size_t)n_levels * n_blocks * 4;
+    const size_t need = (size_t)n_levels * n_blocks * 8;
     if (need > h->loop_trace_cap) {
       void* q = nullptr;
       CU_TRY(h, cudaMalloc(&q, need * 8));
@@ -1191,26 +1195,25 @@ extern "C" int64_t adit_loop_trace_read(adit_handle* h, int64_t* records, int64_
   CU_TRY(h, cudaSetDevice(h->device));
   CU_TRY(h, cudaDeviceSynchronize());
   const int nl = h->loop_trace_levels, nb = h->loop_trace_blocks, per_step = 3 + 5 * h->loop_trace_layers;
-  std::vector<unsigned long long> buf((size_t)nl * nb * 4);
+  std::vector<unsigned long long> buf((size_t)nl * nb * 8);
   CU_TRY(h, cudaMemcpy(buf.data(), h->loop_trace, buf.size() * 8, cudaMemcpyDeviceToHost));
   int64_t n = 0;
   for (int lv = 0; lv < nl && n < max_records; ++lv, ++n) {
     const int j = lv % per_step;
     const int type = j == 0 ? loop::LV_EMBED_IN : j == 1 ? loop::LV_W2 : j == per_step - 1 ? loop::LV_FINAL : loop::LV_QKV + (j - 2) % 5;
-    unsigned long long s_min = ~0ull, s_max = 0, a_max = 0, x_max = 0, e_max = 0;
+    unsigned long long s_min = ~0ull, mx[8] = {0, 0, 0, 0, 0, 0, 0, 0};
     int blocks = 0;
     for (int b = 0; b < nb; ++b) {
-      const unsigned long long* t = &buf[((size_t)lv * nb + b) * 4];
+      const unsigned long long* t = &buf[((size_t)lv * nb + b) * 8];
       if (!t[0]) continue;
       ++blocks;
       if (t[0] < s_min) s_min = t[0];
-      if (t[0] > s_max) s_max = t[0];
-      if (t[1] > a_max) a_max = t[1];
-      if (t[2] > x_max) x_max = t[2];
-      if (t[3] > e_max) e_max = t[3];
+      for (int k = 0; k < 8; ++k)
+        if (t[k] > mx[k]) mx[k] = t[k];
     }
-    int64_t* o = records + n * 7;
-    o[0] = type; o[1] = blocks; o[2] = blocks ? (int64_t)s_min : 0; o[3] = (int64_t)s_max; o[4] = (int64_t)a_max; o[5] = (int64_t)x_max; o[6] = (int64_t)e_max;
+    int64_t* o = records + n * 11;
+    o[0] = type; o[1] = blocks; o[2] = blocks ? (int64_t)s_min : 0;
+    for (int k = 0; k < 8; ++k) o[3 + k] = (int64_t)mx[k];
   }
   return n;
 }

@@ -13,23 +13,23 @@
 //     when its part of a level is stored, the consumers poll with acquire semantics (one polling thread
 //     per block), bounded by a time limit;
 //   * a projection level is cut into cluster units: nf feature tiles x ks k-slices = 8 blocks.  Each block
-//     multiplies its k-slice (tcgen05, accumulator in tensor memory: lane = feature, column = token), pushes
-//     the partial sums straight from registers into the shared memory of the block that owns the token
-//     (st.async over distributed shared memory, counted on the owner's mbarrier), and the owner adds the
-//     ks partials in slice order - bitwise reproducible, independent of the grid size - and runs the fused
-//     epilogue (1/rms scale, GeGLU, residual + bf16 copy + sums of squares for the next norm);
+//     multiplies its k-slice (tcgen05, accumulator in tensor memory: lane = feature, column = token), writes the
+//     partial sums to a per-cluster scratch in global memory (it stays in L2), signals the cluster's blocks through
+//     their mbarriers, and the block that owns a token adds the ks partials in slice order - bitwise reproducible,
+//     independent of the grid size - and runs the fused epilogue (1/rms scale, GeGLU, residual + bf16 copy + sums of
+//     squares for the next norm);
 //   * an attention level is cut into units of (request, kv head, 128 query rows); the 8 blocks of a cluster
 //     take 8 ranges of 64-key blocks (prefix keys padded to a multiple of 64 with masked, zero-filled rows,
 //     then the suffix keys), K/V and Q tiles come in by TMA (prefix blocks before the level's flag: they do
-//     not depend on the step), and the split results are merged inside the cluster: every row's
-//     unnormalised partial goes to the block that owns the row, which combines the 8 splits in fixed order;
+//     not depend on the step), and the split results are merged inside the cluster the same way: every row's
+//     unnormalised partial goes to the scratch, the block that owns the row combines the 8 splits in fixed order;
 //   * the per-step element-wise work (first embedding layer, read-out + Euler update) are levels of their
 //     own, spread over all blocks.
 //
 // Warp roles (256 threads): 0 = weight producer / K,V loader, 1 = flag poller + activation / Q loader,
 // 2 = MMA issuer (projections, Q K^T), 3 = TMEM owner + P V issuer, 4-7 = epilogue / softmax.
-// Shared memory (227 KB): projections see [6 weight slots | 8 activation slots | 64 KB exchange buffer],
-// attention sees [K ring + P | Q | V ring] in the same bytes; a block never runs both at once, and the
+// Shared memory (227 KB): projections see [10 weight slots | 8 activation slots],
+// attention sees [K ring | P | V ring | Q] in the same bytes; a block never runs both at once, and the
 // weight producer drains its ring before an attention unit.  Every wait is bounded.
 #pragma once
 #include "attention.cuh"
@@ -42,20 +42,24 @@ namespace loop {
 
 constexpr int CS = 8;           // blocks per cluster
 constexpr int TOK = 64;         // token tile (MMA N); the path serves at most this many suffix tokens
-constexpr int NSW = 6;          // weight slots of 128 features x 64 k (16 KB)
+constexpr int NSW = 10;         // weight slots of 128 features x 64 k (16 KB)
 constexpr int W_SLOT = 16384;
 constexpr int NSA = 8;          // activation slots of 64 tokens x 64 k (8 KB)
 constexpr int A_SLOT = 8192;
 constexpr int OFF_W = 0;
-constexpr int OFF_A = NSW * W_SLOT;            // 96 KB
-constexpr int OFF_X = OFF_A + NSA * A_SLOT;    // 160 KB
-constexpr int X_BYTES = 65536;
-constexpr int POOL = OFF_X + X_BYTES;          // 224 KB
+constexpr int OFF_A = NSW * W_SLOT;            // 160 KB
+constexpr int POOL = OFF_A + NSA * A_SLOT;     // 224 KB
 // attention view of the same pool
 constexpr int OFF_K = 0;                       // 2 stages of 64 keys x dh (<= 64 KB)
 constexpr int OFF_P = 65536;                   // 2 x [128 rows][64 keys] bf16 (32 KB)
-constexpr int OFF_Q = OFF_A;                   // 128 rows x dh (<= 64 KB); later the merge's receive buffer
-constexpr int OFF_V = OFF_X;                   // 2 stages (<= 64 KB)
+constexpr int OFF_V = 98304;                   // 2 stages (<= 64 KB)
+constexpr int OFF_Q = OFF_A;                   // 128 rows x dh (<= 64 KB)
+// Partial sums of a cluster travel through global memory (L2): per cluster, per source block either
+// [gate | up][64 tokens][128 features] fp32 or [128 rows][dh] bf16 + [128] (max, sum) pairs.  (Distributed shared
+// memory moves about 13 GB/s per block on this part; the same bytes through L2 take a fraction of that time.)
+constexpr int XS_BLOCK_BYTES = 2 * TOK * 128 * 4;                  // 64 KB per source block
+constexpr int XS_ML_OFF = CS * XS_BLOCK_BYTES;                     // (max, sum) pairs after the partials
+constexpr int XS_CLUSTER_BYTES = XS_ML_OFF + CS * 128 * 8;         // 520 KB per cluster
 constexpr int MISC_BYTES = 3072;
 constexpr int SMEM_BYTES = POOL + MISC_BYTES;  // 232448 = the per-block maximum
 constexpr int THREADS = 256;
@@ -92,22 +96,24 @@ struct LoopParams {
   bf16 *hb, *qkv, *att, *mlp, *ez;
   const float *Wfold, *bfold, *ctime, *hs, *ssq_state, *Wout, *bout, *b2;
   const bf16* hsb;
+  uint8_t* xscratch;   // n_clusters x XS_CLUSTER_BYTES
   uint32_t* counters;  // [LV_COUNT] level counters, [LV_COUNT] abort word; zeroed before every call
   int* status;         // host-visible status word
   unsigned long long timeout_ns;
   int debug_skip_level;  // test aid: the level type whose first flag increment of block 0 is withheld (-1: none)
-  unsigned long long* trace;  // optional [level][block][4] timestamps
+  unsigned long long* trace;  // optional [level][block][8] timestamps
 };
 
 struct Misc {
   uint64_t wfull[NSW], wempty[NSW], afull[NSA], aempty[NSA];
   uint64_t acc_full, unit_done, level_go, xfull, xfree;
   uint64_t k_full[2], k_empty[2], v_full[2], v_empty[2], s_full[2], s_empty[2], p_full[2], pv_done[2];
-  uint64_t q_full, xo_ready, xo_full, epi_bar;
+  uint64_t q_full, epi_bar;
   uint32_t tmem_base;
   volatile int abort;
-  float red[4 * 32];
-  float2 ml[CS * 16];  // attention merge: (reference maximum, row sum) per source block and owned row
+  volatile int level_seen;  // participating levels whose dependency the polling thread has observed
+  volatile int units_done;  // units this block's epilogue warps have finished
+  float red[4];
 };
 static_assert(sizeof(Misc) <= MISC_BYTES, "misc region too small");
 
@@ -130,38 +136,64 @@ __device__ __noinline__ void fail(const Ctx& c) {
   atomicExch(c.p->counters + LV_COUNT, 1u);
   c.ms->abort = 1;
 }
-template <bool CLUSTER = false>
+// Waiting must not starve the warps that work: a tight polling loop on a shared-memory barrier fills the memory
+// pipeline that the epilogue's loads and stores and the tensor-core issue go through.  Waits that are expected to be
+// long (ring space, the end of a unit) use the suspending try_wait; waits on the critical path of a level poll the
+// non-blocking test with a short sleep in between.
+__device__ __forceinline__ void nap(unsigned ns) { asm volatile("nanosleep.u32 %0;" ::"r"(ns)); }
+template <bool CRITICAL = true>
 __device__ __forceinline__ bool bwait(const Ctx& c, uint64_t* bar, uint32_t parity) {
-  if (CLUSTER ? ptx::mbar_try_wait_cluster(bar, parity) : ptx::mbar_try_wait(bar, parity)) return true;
+  if (ptx::mbar_test_wait(bar, parity)) return true;
   const uint64_t t0 = ptx::globaltimer_ns();
   for (;;) {
 #pragma unroll 1
-    for (int i = 0; i < 256; ++i)
-      if (CLUSTER ? ptx::mbar_try_wait_cluster(bar, parity) : ptx::mbar_try_wait(bar, parity)) return true;
+    for (int i = 0; i < 512; ++i) {
+      if (CRITICAL) {
+        nap(20);
+        if (ptx::mbar_test_wait(bar, parity)) return true;
+      } else {
+        if (ptx::mbar_try_wait(bar, parity)) return true;
+      }
+    }
     if (gave_up(c, t0)) return false;
   }
 }
-// Whole-warp wait: lane 0 waits with the limit, the others follow.
-template <bool CLUSTER = false>
+// Whole-warp wait: lane 0 waits, the others rejoin at the shuffle.
 __device__ __forceinline__ bool warp_wait(const Ctx& c, uint64_t* bar, uint32_t parity) {
-  const int lane = threadIdx.x & 31;
-  if (__all_sync(0xffffffffu, CLUSTER ? ptx::mbar_try_wait_cluster(bar, parity) : ptx::mbar_test_wait(bar, parity))) return true;
   int okw = 1;
-  if (lane == 0) okw = bwait<CLUSTER>(c, bar, parity) ? 1 : 0;
+  if ((threadIdx.x & 31) == 0) okw = bwait<true>(c, bar, parity) ? 1 : 0;
   okw = __shfl_sync(0xffffffffu, okw, 0);
   if (!okw) return false;
-  for (int spin = 0; spin < 4096 && !(CLUSTER ? ptx::mbar_try_wait_cluster(bar, parity) : ptx::mbar_try_wait(bar, parity)); ++spin) {}
+  // (every lane performs the acquiring test itself; the phase is complete, so this does not spin)
+  while (!ptx::mbar_test_wait(bar, parity)) {}
+  return true;
+}
+// Wait on a count in shared memory that only grows.  A thread that runs ahead of the others by several phases
+// (the weight producer) cannot wait on an mbarrier parity, which only tells neighbouring phases apart.
+__device__ __forceinline__ bool wait_count(const Ctx& c, const volatile int* v, int target) {
+  if (*v >= target) { __threadfence_block(); return true; }
+  const uint64_t t0 = ptx::globaltimer_ns();
+  int spins = 0;
+  while (*v < target) {
+    nap(40);
+    if ((++spins & 255) == 0 && gave_up(c, t0)) return false;
+  }
+  __threadfence_block();
   return true;
 }
 __device__ __forceinline__ bool poll_counter(const Ctx& c, const uint32_t* cnt, uint32_t target) {
-  if (ptx::ld_acquire_gpu(cnt) >= target) return true;
-  const uint64_t t0 = ptx::globaltimer_ns();
-  for (;;) {
+  // relaxed polls (an acquire per poll costs a fence each time), one acquire fence once the count is there
+  bool seen = ptx::ld_relaxed_gpu(cnt) >= target;
+  if (!seen) {
+    const uint64_t t0 = ptx::globaltimer_ns();
+    while (!seen) {
 #pragma unroll 1
-    for (int i = 0; i < 32; ++i)
-      if (ptx::ld_acquire_gpu(cnt) >= target) return true;
-    if (gave_up(c, t0)) return false;
+      for (int i = 0; i < 64 && !seen; ++i) seen = ptx::ld_relaxed_gpu(cnt) >= target;
+      if (!seen && gave_up(c, t0)) return false;
+    }
   }
+  ptx::fence_acq_rel_gpu();
+  return true;
 }
 // Barrier of the four epilogue warps on an mbarrier, so that it is bounded like every other wait: a warp that gave
 // up never arrives and the others leave through the time limit / abort flag instead of hanging in bar.sync.
@@ -269,9 +301,9 @@ __device__ void role_weights(const Ctx& c) {
         for (int j = 0; j < NSW && ok; ++j) {
           const int s = (wslot + j) % NSW;
           const uint32_t ph = (wslot + j >= NSW) ? (wphase ^ 1u) : wphase;
-          if (!bwait(c, &ms->wempty[s], ph ^ 1u)) ok = false;
+          if (!bwait<false>(c, &ms->wempty[s], ph ^ 1u)) ok = false;
         }
-        if (ok && nreal > 0 && !bwait(c, &ms->unit_done, (uint32_t)(nreal - 1) & 1u)) ok = false;
+        if (ok && !wait_count(c, &ms->units_done, nreal)) ok = false;
         if (!ok) break;
         const AttUnit a = att_unit(p, u, c.rank);
         bool flag_seen = false;
@@ -293,7 +325,8 @@ __device__ void role_weights(const Ctx& c) {
               ptx::tma_load_3d(vd + j * (attn::KEY_BLOCK * 128), &p.pk[a.b], j * 64, blk * attn::KEY_BLOCK, plane_v, &ms->v_full[st]);
           } else {
             if (!flag_seen) {  // the suffix keys are this step's: wait for the level's flag (seen by the polling thread)
-              if (!bwait(c, &ms->level_go, (uint32_t)(nlv - 1) & 1u)) { ok = false; break; }
+              // (this thread runs ahead of the levels: a count, not the level barrier's parity)
+              if (!wait_count(c, &ms->level_seen, nlv)) { ok = false; break; }
               ptx::fence_proxy_async_all();
               flag_seen = true;
             }
@@ -309,7 +342,7 @@ __device__ void role_weights(const Ctx& c) {
           }
         }
         // no weight may land in these bytes before the unit is over
-        if (ok && !bwait(c, &ms->unit_done, (uint32_t)nreal & 1u)) ok = false;
+        if (ok && !wait_count(c, &ms->units_done, nreal + 1)) ok = false;
         ++nreal;
       } else {
         const int gi = level_gemm(lv.type);
@@ -320,7 +353,7 @@ __device__ void role_weights(const Ctx& c) {
         const int nv = g.dual ? 2 : 1;
         for (int i = 0; i < g.kbn && ok; ++i) {
           for (int v = 0; v < nv; ++v) {
-            if (!bwait(c, &ms->wempty[wslot], wphase ^ 1u)) { ok = false; break; }
+            if (!bwait<false>(c, &ms->wempty[wslot], wphase ^ 1u)) { ok = false; break; }
             ptx::mbar_arrive_expect_tx(&ms->wfull[wslot], W_SLOT);
             ptx::tma_load_2d_hint(c.pool + OFF_W + wslot * W_SLOT, mw, (gu.sl * g.kbn + i) * 64, gu.ft * 128 * nv + v * 128,
                                   &ms->wfull[wslot], pol);
@@ -342,13 +375,15 @@ __device__ void role_acts(const Ctx& c) {
   const int C = p.n_clusters;
   int aslot = 0; uint32_t aphase = 0;
   uint32_t q_cnt = 0;
-  int nreal = 0;
+  int nreal = 0, nlv = 0;
   bool ok = true;
   const int G = p.n_q_heads / p.n_kv_heads;
   walk_levels(p, [&](const Lv& lv) {
     if (!ok || !participates(lv, c.cid, C)) return;
     if (lv.dep >= 0 && !poll_counter(c, p.counters + lv.dep, lv.dep_target)) { ok = false; return; }
     ptx::fence_proxy_async_all();
+    ms->level_seen = ++nlv;
+    __threadfence_block();
     ptx::mbar_arrive(&ms->level_go);
     if (lv.units == 0) return;
     for (int u = first_unit(lv, c.cid, C); u < lv.units && ok; u += C) {
@@ -358,9 +393,9 @@ __device__ void role_acts(const Ctx& c) {
         for (int j = 0; j < NSA && ok; ++j) {
           const int s = (aslot + j) % NSA;
           const uint32_t ph = (aslot + j >= NSA) ? (aphase ^ 1u) : aphase;
-          if (!bwait(c, &ms->aempty[s], ph ^ 1u)) ok = false;
+          if (!bwait<false>(c, &ms->aempty[s], ph ^ 1u)) ok = false;
         }
-        if (ok && nreal > 0 && !bwait(c, &ms->unit_done, (uint32_t)(nreal - 1) & 1u)) ok = false;
+        if (ok && nreal > 0 && !bwait<false>(c, &ms->unit_done, (uint32_t)(nreal - 1) & 1u)) ok = false;
         if (!ok) break;
         if (a.kb1 > a.kb0) {
           ptx::mbar_arrive_expect_tx(&ms->q_full, 128 * DH * 2);
@@ -375,7 +410,7 @@ __device__ void role_acts(const Ctx& c) {
         if (!gu.valid) continue;
         const CUtensorMap* ma = p.maps + g.map_a;
         for (int i = 0; i < g.kbn; ++i) {
-          if (!bwait(c, &ms->aempty[aslot], aphase ^ 1u)) { ok = false; break; }
+          if (!bwait<false>(c, &ms->aempty[aslot], aphase ^ 1u)) { ok = false; break; }
           ptx::mbar_arrive_expect_tx(&ms->afull[aslot], A_SLOT);
           ptx::tma_load_2d(c.pool + OFF_A + aslot * A_SLOT, ma, (gu.sl * g.kbn + i) * 64, 0, &ms->afull[aslot]);
           if (++aslot == NSA) { aslot = 0; aphase ^= 1u; }
@@ -400,6 +435,7 @@ __device__ void role_mma(const Ctx& c) {
   int nreal = 0;
   bool ok = true;
   const uint32_t idesc = ptx::idesc_bf16_f32(128, TOK);
+  const uint64_t wdesc0 = ptx::smem_desc_sw128(ptx::smem_u32(c.pool + OFF_W)), adesc0 = ptx::smem_desc_sw128(ptx::smem_u32(c.pool + OFF_A));
   const uint32_t idesc_s = ptx::idesc_bf16_f32(128, attn::KEY_BLOCK);
   const uint32_t tm_s = c.tmem + 256;
   walk_levels(p, [&](const Lv& lv) {
@@ -408,7 +444,7 @@ __device__ void role_mma(const Ctx& c) {
       if (lv.type == LV_ATT) {
         const AttUnit a = att_unit(p, u, c.rank);
         const int nb = a.kb1 - a.kb0;
-        if (nreal > 0 && !bwait(c, &ms->unit_done, (uint32_t)(nreal - 1) & 1u)) { ok = false; break; }
+        if (nreal > 0 && !bwait<false>(c, &ms->unit_done, (uint32_t)(nreal - 1) & 1u)) { ok = false; break; }
         if (nb > 0) {
           if (!bwait(c, &ms->q_full, q_cnt & 1u)) { ok = false; break; }
           ++q_cnt;
@@ -431,20 +467,24 @@ __device__ void role_mma(const Ctx& c) {
         const GemmLv& g = p.g[level_gemm(lv.type)];
         const GemmUnit gu = gemm_unit(g, u, c.rank);
         if (!gu.valid) continue;
-        if (nreal > 0 && !bwait(c, &ms->unit_done, (uint32_t)(nreal - 1) & 1u)) { ok = false; break; }
+        if (nreal > 0 && !bwait<false>(c, &ms->unit_done, (uint32_t)(nreal - 1) & 1u)) { ok = false; break; }
         ptx::tc_fence_after();
         const int nv = g.dual ? 2 : 1;
+        unsigned long long* tr = p.trace ? p.trace + ((size_t)lv.seq * c.n_cta + c.cta) * 8 : nullptr;
         for (int i = 0; i < g.kbn && ok; ++i) {
           if (!bwait(c, &ms->afull[aslot], aphase)) { ok = false; break; }
-          const uint32_t as = ptx::smem_u32(c.pool + OFF_A + aslot * A_SLOT);
+          if (tr && i == 0) tr[6] = ptx::globaltimer_ns();
+          // descriptors differ from the first slot's only in the start-address field (16-byte units)
+          const uint64_t ad = adesc0 + (uint64_t)(aslot * (A_SLOT >> 4));
           for (int v = 0; v < nv; ++v) {
             if (!bwait(c, &ms->wfull[wslot], wphase)) { ok = false; break; }
             ptx::tc_fence_after();
-            const uint32_t ws = ptx::smem_u32(c.pool + OFF_W + wslot * W_SLOT);
-#pragma unroll
-            for (int k4 = 0; k4 < 4; ++k4)
-              ptx::umma_f16(c.tmem + (uint32_t)(v * TOK), ptx::smem_desc_sw128(ws + k4 * 32), ptx::smem_desc_sw128(as + k4 * 32), idesc,
-                            (i > 0 || k4 > 0) ? 1u : 0u);
+            const uint64_t wd = wdesc0 + (uint64_t)(wslot * (W_SLOT >> 4));
+            const uint32_t d = c.tmem + (uint32_t)(v * TOK);
+            ptx::umma_f16(d, wd, ad, idesc, i > 0 ? 1u : 0u);
+            ptx::umma_f16(d, wd + 2, ad + 2, idesc, 1u);
+            ptx::umma_f16(d, wd + 4, ad + 4, idesc, 1u);
+            ptx::umma_f16(d, wd + 6, ad + 6, idesc, 1u);
             ptx::umma_commit(&ms->wempty[wslot]);
             if (++wslot == NSW) { wslot = 0; wphase ^= 1u; }
           }
@@ -452,6 +492,7 @@ __device__ void role_mma(const Ctx& c) {
           if (++aslot == NSA) { aslot = 0; aphase ^= 1u; }
         }
         if (ok) ptx::umma_commit(&ms->acc_full);
+        if (tr) tr[7] = ptx::globaltimer_ns();
         ++nreal;
       }
     }
@@ -480,7 +521,7 @@ __device__ void role_pv(const Ctx& c) {
       }
       const AttUnit a = att_unit(p, u, c.rank);
       const int nb = a.kb1 - a.kb0;
-      if (nreal > 0 && !bwait(c, &ms->unit_done, (uint32_t)(nreal - 1) & 1u)) { ok = false; break; }
+      if (nreal > 0 && !bwait<false>(c, &ms->unit_done, (uint32_t)(nreal - 1) & 1u)) { ok = false; break; }
       for (int i = 0; i < nb; ++i, ++kv_cnt) {
         const int s = kv_cnt & 1;
         const uint32_t par = (kv_cnt >> 1) & 1u;
@@ -532,13 +573,20 @@ __device__ void level_embed_in(const Ctx& c, const Lv& lv, int et) {
       const float bias = p.bfold[col] + cvec[col];
       float acc[4] = {bias, bias, bias, bias};
       const float* wr = p.Wfold + (int64_t)col * p.A;
-      for (int j = 0; j < p.A; ++j) {
-        const float w = __ldg(wr + j);
+      // eight inputs per pass so that the loads of a pass are in flight together
+      for (int j0 = 0; j0 < p.A; j0 += 8) {
+        float w[8], xv[4][8];
 #pragma unroll
-        for (int r = 0; r < 4; ++r) {
-          const int m = min(m0 + r, p.Ma - 1);
-          acc[r] = fmaf(__ldcg(p.x + (int64_t)m * p.A + j), w, acc[r]);
+        for (int j = 0; j < 8; ++j) {
+          const int jj = min(j0 + j, p.A - 1);
+          w[j] = j0 + j < p.A ? __ldg(wr + jj) : 0.f;
+#pragma unroll
+          for (int r = 0; r < 4; ++r) xv[r][j] = __ldcg(p.x + (int64_t)min(m0 + r, p.Ma - 1) * p.A + jj);
         }
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+#pragma unroll
+          for (int r = 0; r < 4; ++r) acc[r] = fmaf(xv[r][j], w[j], acc[r]);
       }
 #pragma unroll
       for (int r = 0; r < 4; ++r)
@@ -569,6 +617,7 @@ __device__ bool level_final(const Ctx& c, const Lv& lv, int et, int& nsync) {
     const float4* row = reinterpret_cast<const float4*>(p.h + ((int64_t)m + m / p.horizon + 1) * p.D);
     float ss = 0.f;
     if (!epi_sync(c, nsync)) return false;
+#pragma unroll 2
     for (int d = et; d < p.D / 4; d += 128) {
       const float4 v = __ldcg(row + d);
       srow[d] = v;
@@ -582,6 +631,7 @@ __device__ bool level_final(const Ctx& c, const Lv& lv, int et, int& nsync) {
     for (int j = part * per_part + ew; j < j_end; j += 4) {
       const float4* wr = reinterpret_cast<const float4*>(p.Wout + (int64_t)j * p.D);
       float a = 0.f;
+#pragma unroll 4
       for (int d = lane; d < p.D / 4; d += 32) {
         const float4 w4 = __ldg(wr + d), v = srow[d];
         a = fmaf(v.x, w4.x, a); a = fmaf(v.y, w4.y, a); a = fmaf(v.z, w4.z, a); a = fmaf(v.w, w4.w, a);
@@ -597,6 +647,115 @@ __device__ bool level_final(const Ctx& c, const Lv& lv, int et, int& nsync) {
   return true;
 }
 
+
+// Signal "this warp's partial sums are in the scratch" to every block of the cluster (one arrival per warp and
+// block on each xfull barrier): a cluster-scope fence after the warp's stores, then relaxed remote arrivals.
+__device__ __forceinline__ void signal_partials(const Ctx& c) {
+  __syncwarp();
+  if ((threadIdx.x & 31) == 0) {
+    asm volatile("fence.acq_rel.cluster;" ::: "memory");
+    const uint32_t bar = ptx::smem_u32(&c.ms->xfull);
+    for (int r = 0; r < CS; ++r) ptx::mbar_arrive_remote_relaxed(ptx::mapa_shared(bar, r));
+  }
+}
+// Wait for all partial sums of the cluster's current unit (acquire at cluster scope once the phase is complete).
+__device__ __forceinline__ bool wait_partials(const Ctx& c, uint32_t parity) {
+  if (!warp_wait(c, &c.ms->xfull, parity)) return false;
+  asm volatile("fence.acq_rel.cluster;" ::: "memory");
+  return true;
+}
+__device__ __forceinline__ void release_scratch(const Ctx& c, int et) {
+  if (et == 0) {
+    const uint32_t bar = ptx::smem_u32(&c.ms->xfree);
+    for (int r = 0; r < CS; ++r) ptx::mbar_arrive_remote_relaxed(ptx::mapa_shared(bar, r));
+  }
+}
+__device__ __forceinline__ float4 f4add(float4 a, float4 b) { return make_float4(a.x + b.x, a.y + b.y, a.z + b.z, a.w + b.w); }
+
+// Second half of a projection unit's epilogue.  This block owns tpo = 64 / ks tokens of the tile; warp w takes the
+// tokens my_tok0 + w, + 4, ... (tpw = tpo / 4 of them), lane q the features 4q .. 4q + 3.  Every value is the sum of
+// the ks partials in slice order; tpw * ks = 16 loads per lane (and gate/up part) are in flight together.
+template <int NV>
+__device__ __forceinline__ void finalize_owned(const Ctx& c, const GemmLv& g, const GemmUnit& gu, int n_tok_valid, int lane, int ew,
+                                               const float4 (&old4)[8], float rs_lane) {
+  const LoopParams& p = *c.p;
+  const int tpo = TOK / g.ks, tpw = tpo >> 2, my_tok0 = gu.sl * tpo;
+  const float* xs = reinterpret_cast<const float*>(p.xscratch + (size_t)c.cid * XS_CLUSTER_BYTES);
+  const int ksh = g.ks == 8 ? 3 : g.ks == 4 ? 2 : 1;
+  float4 buf[16 * NV];
+#pragma unroll
+  for (int i = 0; i < 16; ++i) {
+    const int t = i >> ksh, sl = i & (g.ks - 1);  // token slot, source slice
+    const int tok = my_tok0 + ew + 4 * t;
+    const int src = gu.grp * g.ks + sl;
+#pragma unroll
+    for (int vv = 0; vv < NV; ++vv)
+      buf[i * NV + vv] = tok < n_tok_valid ? __ldcg(reinterpret_cast<const float4*>(xs + ((size_t)((src * 2 + vv) * TOK + tok)) * 128) + lane)
+                                           : make_float4(0.f, 0.f, 0.f, 0.f);
+  }
+  float4 sum[8 * NV];
+  if (g.ks == 8) {
+#pragma unroll
+    for (int t = 0; t < 2; ++t)
+#pragma unroll
+      for (int vv = 0; vv < NV; ++vv) {
+        float4 a = buf[(t * 8) * NV + vv];
+#pragma unroll
+        for (int q = 1; q < 8; ++q) a = f4add(a, buf[(t * 8 + q) * NV + vv]);
+        sum[t * NV + vv] = a;
+      }
+  } else if (g.ks == 4) {
+#pragma unroll
+    for (int t = 0; t < 4; ++t)
+#pragma unroll
+      for (int vv = 0; vv < NV; ++vv) {
+        float4 a = buf[(t * 4) * NV + vv];
+#pragma unroll
+        for (int q = 1; q < 4; ++q) a = f4add(a, buf[(t * 4 + q) * NV + vv]);
+        sum[t * NV + vv] = a;
+      }
+  } else {
+#pragma unroll
+    for (int t = 0; t < 8; ++t)
+#pragma unroll
+      for (int vv = 0; vv < NV; ++vv) sum[t * NV + vv] = f4add(buf[(t * 2) * NV + vv], buf[(t * 2 + 1) * NV + vv]);
+  }
+  const int col = gu.ft * 128 + 4 * lane;
+  float4 bias4 = make_float4(0.f, 0.f, 0.f, 0.f);
+  if (g.epi == LEPI_EMBED) bias4 = *reinterpret_cast<const float4*>(p.b2 + col);
+#pragma unroll
+  for (int t = 0; t < 8; ++t) {
+    if (t < tpw) {
+      const int tok = my_tok0 + ew + 4 * t;
+      const bool tv = tok < n_tok_valid;
+      const float4 v = sum[t * NV];
+      if (g.epi == LEPI_STORE) {
+        const float r = __shfl_sync(0xffffffffu, rs_lane, t);
+        if (tv) *reinterpret_cast<uint2*>(p.qkv + (int64_t)tok * g.ldo + col) = make_uint2(attn::pack_bf16(v.x * r, v.y * r), attn::pack_bf16(v.z * r, v.w * r));
+      } else if (g.epi == LEPI_GEGLU) {
+        const float r = __shfl_sync(0xffffffffu, rs_lane, t);
+        const float4 u = sum[t * NV + (NV - 1)];
+        if (tv)
+          *reinterpret_cast<uint2*>(p.mlp + (int64_t)tok * g.ldo + col) =
+              make_uint2(attn::pack_bf16(tc::gelu_tanh_fast(v.x * r) * (u.x * r), tc::gelu_tanh_fast(v.y * r) * (u.y * r)),
+                         attn::pack_bf16(tc::gelu_tanh_fast(v.z * r) * (u.z * r), tc::gelu_tanh_fast(v.w * r) * (u.w * r)));
+      } else {
+        float4 hv;
+        int64_t rowi;
+        if (g.epi == LEPI_RESID) { hv = f4add(old4[t], v); rowi = tok; }
+        else { hv = f4add(v, bias4); rowi = tok + tok / p.horizon + 1; }
+        float sq = (hv.x * hv.x + hv.y * hv.y) + (hv.z * hv.z + hv.w * hv.w);
+        for (int o = 16; o; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
+        if (tv) {
+          *reinterpret_cast<float4*>(p.h + rowi * p.D + col) = hv;
+          *reinterpret_cast<uint2*>(p.hb + rowi * p.D + col) = make_uint2(attn::pack_bf16(hv.x, hv.y), attn::pack_bf16(hv.z, hv.w));
+          if (lane == 0) p.ssq[(int64_t)gu.ft * p.ssq_ld + rowi] = sq;
+        }
+      }
+    }
+  }
+}
+
 // ---- role: epilogue of the projections, softmax of the attention, element-wise levels ---------------
 template <int DH>
 __device__ void role_epilogue(const Ctx& c) {
@@ -610,7 +769,7 @@ __device__ void role_epilogue(const Ctx& c) {
   const uint32_t lane_addr = (uint32_t)(ew * 32) << 16;
   const int G = p.n_q_heads / p.n_kv_heads, R = p.n_tok * G;
   const uint32_t tm_s = c.tmem + 256;
-  int nlv = 0, nreal = 0, ngemm = 0, nxch = 0, natt = 0, nsync = 0;
+  int nlv = 0, nreal = 0, ngemm = 0, nx = 0, nsync = 0;
   uint32_t kv_cnt = 0;
   uint32_t seen_types = 0;  // level types this block has published at least once
   bool ok = true;
@@ -618,15 +777,16 @@ __device__ void role_epilogue(const Ctx& c) {
     if (!ok || !participates(lv, c.cid, C)) return;
     if (!warp_wait(c, &ms->level_go, (uint32_t)nlv & 1u)) { ok = false; return; }
     ++nlv;
-    unsigned long long* tr = (p.trace && et == 0) ? p.trace + ((size_t)lv.seq * c.n_cta + c.cta) * 4 : nullptr;
+    unsigned long long* tr = (p.trace && et == 0) ? p.trace + ((size_t)lv.seq * c.n_cta + c.cta) * 8 : nullptr;
     if (tr) tr[0] = ptx::globaltimer_ns();
     const bool first_of_type = !((seen_types >> lv.type) & 1u);
     seen_types |= 1u << lv.type;
     if (lv.units == 0) {
+      if (tr) { tr[1] = (unsigned long long)clock64(); tr[2] = ptx::globaltimer_ns(); }
       if (lv.type == LV_EMBED_IN) level_embed_in(c, lv, et);
       else if (!level_final(c, lv, et, nsync)) { ok = false; return; }
       if (!publish(c, lv.type, et, first_of_type, nsync)) { ok = false; return; }
-      if (tr) tr[3] = ptx::globaltimer_ns();
+      if (tr) { tr[3] = (unsigned long long)clock64(); tr[5] = ptx::globaltimer_ns(); }
       return;
     }
     bool first_unit_of_level = true;
@@ -636,7 +796,6 @@ __device__ void role_epilogue(const Ctx& c) {
         const AttUnit a = att_unit(p, u, c.rank);
         const int nb = a.kb1 - a.kb0;
         const int row = et;
-        if (et == 0) ptx::mbar_arrive_expect_tx(&ms->xo_full, (uint32_t)(CS * 16 * (DH * 2 + 8)));
         float m_ref = -INFINITY, l = 0.f;
         for (int i = 0; i < nb && ok; ++i) {
           const uint32_t n = kv_cnt + i;
@@ -721,20 +880,12 @@ __device__ void role_epilogue(const Ctx& c) {
         }
         kv_cnt += nb;
         if (tr && first_unit_of_level) tr[1] = ptx::globaltimer_ns();
-        // ---- merge of the 8 key ranges inside the cluster ----
-        // All of this block's products are complete: its Q tile may now be overwritten by the peers' rows.
-        if (!epi_sync(c, nsync)) { ok = false; break; }
-        if (et == 0) {
-          const uint32_t bar = ptx::smem_u32(&ms->xo_ready);
-          for (int r = 0; r < CS; ++r) ptx::mbar_arrive_remote(ptx::mapa_shared(bar, r));
-        }
-        if (!warp_wait<true>(c, &ms->xo_ready, (uint32_t)natt & 1u)) { ok = false; break; }
+        // ---- merge of the 8 key ranges inside the cluster, through the scratch in global memory ----
+        if (nx > 0 && !warp_wait(c, &ms->xfree, (uint32_t)(nx - 1) & 1u)) { ok = false; break; }
         {
-          const int owner = row >> 4, rl = row & 15;
-          const uint32_t dst = ptx::mapa_shared(ptx::smem_u32(c.pool + OFF_Q) + (uint32_t)((c.rank * 16 + rl) * (DH * 2)), owner);
-          const uint32_t bar = ptx::mapa_shared(ptx::smem_u32(&ms->xo_full), owner);
-          const uint32_t mld = ptx::mapa_shared(ptx::smem_u32(&ms->ml[c.rank * 16 + rl]), owner);
-          ptx::st_async_v2(mld, __float_as_uint(m_ref), __float_as_uint(l), bar);
+          uint8_t* xs = p.xscratch + (size_t)c.cid * XS_CLUSTER_BYTES;
+          uint4* dst = reinterpret_cast<uint4*>(xs + (size_t)c.rank * XS_BLOCK_BYTES + (size_t)row * (DH * 2));
+          reinterpret_cast<float2*>(xs + XS_ML_OFF)[c.rank * 128 + row] = make_float2(m_ref, l);
 #pragma unroll 1
           for (int c0 = 0; c0 < DH; c0 += 32) {
             float o[32];
@@ -747,20 +898,26 @@ __device__ void role_epilogue(const Ctx& c) {
             }
 #pragma unroll
             for (int j = 0; j < 32; j += 8)
-              ptx::st_async_v4(dst + (uint32_t)(c0 + j) * 2, attn::pack_bf16(o[j], o[j + 1]), attn::pack_bf16(o[j + 2], o[j + 3]),
-                               attn::pack_bf16(o[j + 4], o[j + 5]), attn::pack_bf16(o[j + 6], o[j + 7]), bar);
+              dst[(c0 + j) >> 3] = make_uint4(attn::pack_bf16(o[j], o[j + 1]), attn::pack_bf16(o[j + 2], o[j + 3]),
+                                              attn::pack_bf16(o[j + 4], o[j + 5]), attn::pack_bf16(o[j + 6], o[j + 7]));
           }
           ptx::tc_fence_before();
         }
-        if (!warp_wait<true>(c, &ms->xo_full, (uint32_t)natt & 1u)) { ok = false; break; }
+        signal_partials(c);
+        if (!wait_partials(c, (uint32_t)nx & 1u)) { ok = false; break; }
         {
           // thread = (owned row, 1/8 of the channels): weights of the 8 ranges in fixed order
           constexpr int CPT = DH / 8;  // channels per thread
           const int rl = et >> 3, part = et & 7;
+          const int rrow = c.rank * 16 + rl;  // row of the tile owned by this block
+          const uint8_t* xs = p.xscratch + (size_t)c.cid * XS_CLUSTER_BYTES;
           float mm[CS], ll[CS];
           float M = -INFINITY;
 #pragma unroll
-          for (int s = 0; s < CS; ++s) { const float2 v = ms->ml[s * 16 + rl]; mm[s] = v.x; ll[s] = v.y; M = fmaxf(M, v.x); }
+          for (int s = 0; s < CS; ++s) {
+            const float2 v = __ldcg(reinterpret_cast<const float2*>(xs + XS_ML_OFF) + s * 128 + rrow);
+            mm[s] = v.x; ll[s] = v.y; M = fmaxf(M, v.x);
+          }
           float L = 0.f;
 #pragma unroll
           for (int s = 0; s < CS; ++s) { mm[s] = mm[s] == -INFINITY ? 0.f : exp2f(mm[s] - M); L += ll[s] * mm[s]; }
@@ -769,20 +926,26 @@ __device__ void role_epilogue(const Ctx& c) {
 #pragma unroll
           for (int e = 0; e < CPT; ++e) acc[e] = 0.f;
 #pragma unroll
-          for (int s = 0; s < CS; ++s) {
-            const uint4* src = reinterpret_cast<const uint4*>(c.pool + OFF_Q + (size_t)((s * 16 + rl) * (DH * 2)) + part * CPT * 2);
+          for (int s0 = 0; s0 < CS; s0 += 4) {
+            uint4 raw[4][CPT / 8];
 #pragma unroll
-            for (int q = 0; q < CPT / 8; ++q) {
-              const uint4 t = src[q];
-              const uint32_t w[4] = {t.x, t.y, t.z, t.w};
+            for (int s = 0; s < 4; ++s)
 #pragma unroll
-              for (int k = 0; k < 4; ++k) {
-                acc[q * 8 + 2 * k] = fmaf(__uint_as_float(w[k] << 16), mm[s], acc[q * 8 + 2 * k]);
-                acc[q * 8 + 2 * k + 1] = fmaf(__uint_as_float(w[k] & 0xffff0000u), mm[s], acc[q * 8 + 2 * k + 1]);
+              for (int q = 0; q < CPT / 8; ++q)
+                raw[s][q] = __ldcg(reinterpret_cast<const uint4*>(xs + (size_t)(s0 + s) * XS_BLOCK_BYTES + (size_t)rrow * (DH * 2) + part * CPT * 2) + q);
+#pragma unroll
+            for (int s = 0; s < 4; ++s)
+#pragma unroll
+              for (int q = 0; q < CPT / 8; ++q) {
+                const uint32_t w[4] = {raw[s][q].x, raw[s][q].y, raw[s][q].z, raw[s][q].w};
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                  acc[q * 8 + 2 * k] = fmaf(__uint_as_float(w[k] << 16), mm[s0 + s], acc[q * 8 + 2 * k]);
+                  acc[q * 8 + 2 * k + 1] = fmaf(__uint_as_float(w[k] & 0xffff0000u), mm[s0 + s], acc[q * 8 + 2 * k + 1]);
+                }
               }
-            }
           }
-          const int gr = a.rt * 128 + c.rank * 16 + rl;
+          const int gr = a.rt * 128 + rrow;
           if (gr < R) {
             const int tok = gr / G, hq = a.kvh * G + (gr - tok * G);
             uint4* dstg = reinterpret_cast<uint4*>(p.att + (int64_t)(a.tok0 + tok) * (p.n_q_heads * DH) + hq * DH + part * CPT);
@@ -792,8 +955,10 @@ __device__ void role_epilogue(const Ctx& c) {
                                    attn::pack_bf16(acc[q * 8 + 4] * inv, acc[q * 8 + 5] * inv), attn::pack_bf16(acc[q * 8 + 6] * inv, acc[q * 8 + 7] * inv));
           }
         }
-        ++natt;
+        ++nx;
         if (!publish(c, LV_ATT, et, first_of_type && first_unit_of_level, nsync)) { ok = false; break; }
+        release_scratch(c, et);
+        if (et == 0) { __threadfence_block(); ms->units_done = nreal + 1; }
         __syncwarp();
         if (lane == 0) ptx::mbar_arrive(&ms->unit_done);
         ++nreal;
@@ -802,48 +967,43 @@ __device__ void role_epilogue(const Ctx& c) {
         const int gi = level_gemm(lv.type);
         const GemmLv& g = p.g[gi];
         const GemmUnit gu = gemm_unit(g, u, c.rank);
-        const uint32_t xfree_bar = ptx::smem_u32(&ms->xfree);
         if (!gu.valid) {  // this block has no tile in the unit: it only keeps the counts going
-          if (et == 0) {
-            for (int r = 0; r < CS; ++r) ptx::mbar_arrive_remote(ptx::mapa_shared(xfree_bar, r));
-          }
+          if (nx > 0 && !warp_wait(c, &ms->xfree, (uint32_t)(nx - 1) & 1u)) { ok = false; break; }
+          signal_partials(c);
+          release_scratch(c, et);
           if (!publish(c, lv.type, et, first_of_type && first_unit_of_level, nsync)) { ok = false; break; }
-          ++nxch;
+          ++nx;
           continue;
         }
         const int nv = g.dual ? 2 : 1;
-        const int tpo = TOK / g.ks;          // tokens finalised by this block
+        const int tpo = TOK / g.ks, tpw = tpo >> 2;  // tokens finalised by this block / by each of its warps
         const int my_tok0 = gu.sl * tpo;
-        const int f = et;                    // feature within the tile = TMEM lane
         const int n_tok_valid = g.epi == LEPI_EMBED ? p.Ma : p.M;
-        if (et == 0) ptx::mbar_arrive_expect_tx(&ms->xfull, (uint32_t)(nv * 128 * TOK * 4));
-        // what does not depend on the accumulator: 1/rms of the owned tokens (lane t: token my_tok0 + t), old residuals
+        // what does not depend on the accumulator: 1/rms of this warp's tokens (lane t: token slot t), old residuals
         float rs_lane = 1.f;
-        if ((g.epi == LEPI_STORE || g.epi == LEPI_GEGLU) && lane < tpo) {
-          const int tok = my_tok0 + lane;
+        if ((g.epi == LEPI_STORE || g.epi == LEPI_GEGLU) && lane < tpw) {
+          const int tok = my_tok0 + ew + 4 * lane;
           if (tok < n_tok_valid) {
             float tot = 0.f;
             for (int i = 0; i < p.n_dtiles; ++i) tot += __ldcg(p.ssq + (int64_t)i * p.ssq_ld + tok);
             rs_lane = 1.0f / sqrtf(tot / (float)p.D + p.eps);
           }
         }
-        float old[32];
-        if (g.epi == LEPI_RESID) {
-          const float* hp = p.h + (int64_t)my_tok0 * p.D + gu.ft * 128 + f;
+        float4 old4[8];
 #pragma unroll
-          for (int j = 0; j < 32; ++j) old[j] = (j < tpo && my_tok0 + j < n_tok_valid) ? __ldcg(hp + (int64_t)j * p.D) : 0.f;
-        } else {
-#pragma unroll
-          for (int j = 0; j < 32; ++j) old[j] = 0.f;
+        for (int t = 0; t < 8; ++t) {
+          const int tok = my_tok0 + ew + 4 * t;
+          old4[t] = (g.epi == LEPI_RESID && t < tpw && tok < n_tok_valid)
+                        ? __ldcg(reinterpret_cast<const float4*>(p.h + (int64_t)tok * p.D + gu.ft * 128) + lane)
+                        : make_float4(0.f, 0.f, 0.f, 0.f);
         }
         if (!warp_wait(c, &ms->acc_full, (uint32_t)ngemm & 1u)) { ok = false; break; }
         ptx::tc_fence_after();
         if (tr && first_unit_of_level) tr[1] = ptx::globaltimer_ns();
-        if (nxch > 0 && !warp_wait<true>(c, &ms->xfree, (uint32_t)(nxch - 1) & 1u)) { ok = false; break; }
-        // push the partial sums to the owners of the tokens: X[source slice][gate | up][feature][owned token]
+        if (nx > 0 && !warp_wait(c, &ms->xfree, (uint32_t)(nx - 1) & 1u)) { ok = false; break; }
+        // partial sums -> scratch[this block][gate | up][token][feature]; thread = feature (TMEM lane)
         {
-          const uint32_t x_local = ptx::smem_u32(c.pool + OFF_X);
-          const uint32_t bar_local = ptx::smem_u32(&ms->xfull);
+          float* xs = reinterpret_cast<float*>(p.xscratch + (size_t)c.cid * XS_CLUSTER_BYTES) + (size_t)c.rank * (2 * TOK * 128) + et;
 #pragma unroll 1
           for (int vv = 0; vv < nv; ++vv) {
 #pragma unroll 1
@@ -851,106 +1011,30 @@ __device__ void role_epilogue(const Ctx& c) {
               float v[32];
               ptx::tmem_ld_32x32(c.tmem + (uint32_t)(vv * TOK + c0) + lane_addr, v);
               ptx::tmem_ld_wait();
-              for (int o = c0 / tpo; o < (c0 + 32) / tpo; ++o) {
-                const int dst_rank = gu.grp * g.ks + o;
-                const uint32_t dst = ptx::mapa_shared(x_local + (uint32_t)(((gu.sl * nv + vv) * 128 + f) * tpo) * 4u, dst_rank);
-                const uint32_t bar = ptx::mapa_shared(bar_local, dst_rank);
-                const int base = o * tpo - c0;
+              float* dst = xs + (size_t)(vv * TOK + c0) * 128;
 #pragma unroll
-                for (int j = 0; j < 32; j += 4)
-                  if (j < tpo) {
-                    // (v is indexed with compile-time offsets per candidate base to stay in registers)
-                    float a0, a1, a2, a3;
-                    if (base == 0) { a0 = v[j]; a1 = v[j + 1]; a2 = v[j + 2]; a3 = v[j + 3]; }
-                    else if (base == 8) { a0 = v[(j + 8) & 31]; a1 = v[(j + 9) & 31]; a2 = v[(j + 10) & 31]; a3 = v[(j + 11) & 31]; }
-                    else if (base == 16) { a0 = v[(j + 16) & 31]; a1 = v[(j + 17) & 31]; a2 = v[(j + 18) & 31]; a3 = v[(j + 19) & 31]; }
-                    else { a0 = v[(j + 24) & 31]; a1 = v[(j + 25) & 31]; a2 = v[(j + 26) & 31]; a3 = v[(j + 27) & 31]; }
-                    ptx::st_async_v4(dst + (uint32_t)j * 4u, __float_as_uint(a0), __float_as_uint(a1), __float_as_uint(a2), __float_as_uint(a3), bar);
-                  }
-              }
+              for (int j = 0; j < 32; ++j)
+                if (c0 + j < n_tok_valid) dst[j * 128] = v[j];
             }
           }
         }
         ptx::tc_fence_before();
-        if (!warp_wait<true>(c, &ms->xfull, (uint32_t)ngemm & 1u)) { ok = false; break; }
+        signal_partials(c);
         if (tr && first_unit_of_level) tr[2] = ptx::globaltimer_ns();
-        // sum the ks partials in slice order, 8 tokens at a time, and finalise
-        const float* X = reinterpret_cast<const float*>(c.pool + OFF_X);
-        const float bias = g.epi == LEPI_EMBED ? p.b2[gu.ft * 128 + f] : 0.f;
-#pragma unroll 1
-        for (int c0 = 0; c0 < tpo; c0 += 8) {
-          float v[8], v2[8];
-#pragma unroll
-          for (int j = 0; j < 8; ++j) { v[j] = 0.f; v2[j] = 0.f; }
-#pragma unroll 1
-          for (int s = 0; s < g.ks; ++s) {
-            const float4* src = reinterpret_cast<const float4*>(X + (size_t)((s * nv) * 128 + f) * tpo + c0);
-            const float4 a0 = src[0], a1 = src[1];
-            v[0] += a0.x; v[1] += a0.y; v[2] += a0.z; v[3] += a0.w; v[4] += a1.x; v[5] += a1.y; v[6] += a1.z; v[7] += a1.w;
-            if (nv == 2) {
-              const float4* src2 = reinterpret_cast<const float4*>(X + (size_t)((s * nv + 1) * 128 + f) * tpo + c0);
-              const float4 b0 = src2[0], b1 = src2[1];
-              v2[0] += b0.x; v2[1] += b0.y; v2[2] += b0.z; v2[3] += b0.w; v2[4] += b1.x; v2[5] += b1.y; v2[6] += b1.z; v2[7] += b1.w;
-            }
-          }
-          float sq[8];
-#pragma unroll
-          for (int j = 0; j < 8; ++j) {
-            const int tok = my_tok0 + c0 + j;
-            const bool tv = tok < n_tok_valid;
-            sq[j] = 0.f;
-            if (g.epi == LEPI_STORE) {
-              const float r = __shfl_sync(0xffffffffu, rs_lane, c0 + j);
-              if (tv) p.qkv[(int64_t)tok * g.ldo + gu.ft * 128 + f] = __float2bfloat16_rn(v[j] * r);
-            } else if (g.epi == LEPI_GEGLU) {
-              const float r = __shfl_sync(0xffffffffu, rs_lane, c0 + j);
-              if (tv) p.mlp[(int64_t)tok * g.ldo + gu.ft * 128 + f] = __float2bfloat16_rn(tc::gelu_tanh_fast(v[j] * r) * (v2[j] * r));
-            } else {
-              float hv;
-              int64_t rowi;
-              if (g.epi == LEPI_RESID) {
-                float o = 0.f;
-#pragma unroll
-                for (int q = 0; q < 32; q += 8)
-                  if (c0 == q) o = old[q + j];
-                hv = o + v[j];
-                rowi = tok;
-              } else {
-                hv = v[j] + bias;
-                rowi = tok + tok / p.horizon + 1;
-              }
-              if (tv) {
-                p.h[rowi * p.D + gu.ft * 128 + f] = hv;
-                p.hb[rowi * p.D + gu.ft * 128 + f] = __float2bfloat16_rn(hv);
-                sq[j] = hv * hv;
-              }
-            }
-          }
-          if (g.epi == LEPI_RESID || g.epi == LEPI_EMBED) {
-            tc::warp_sum_transposed<8>(sq, lane);
-            if ((lane & 3) == 0) ms->red[ew * 32 + c0 + (lane >> 2)] = sq[0];
-          }
-        }
-        if (g.epi == LEPI_RESID || g.epi == LEPI_EMBED) {
-          if (!epi_sync(c, nsync)) { ok = false; break; }
-          if (et < tpo) {
-            const int tok = my_tok0 + et;
-            if (tok < n_tok_valid) {
-              const int64_t rowi = g.epi == LEPI_EMBED ? (tok + tok / p.horizon + 1) : tok;
-              p.ssq[(int64_t)gu.ft * p.ssq_ld + rowi] = ((ms->red[et] + ms->red[32 + et]) + ms->red[64 + et]) + ms->red[96 + et];
-            }
-          }
-        }
+        if (!wait_partials(c, (uint32_t)nx & 1u)) { ok = false; break; }
+        if (tr && first_unit_of_level) tr[3] = ptx::globaltimer_ns();
+        if (nv == 2) finalize_owned<2>(c, g, gu, n_tok_valid, lane, ew, old4, rs_lane);
+        else finalize_owned<1>(c, g, gu, n_tok_valid, lane, ew, old4, rs_lane);
+        if (tr && first_unit_of_level) tr[4] = ptx::globaltimer_ns();
         if (!publish(c, lv.type, et, first_of_type && first_unit_of_level, nsync)) { ok = false; break; }
-        if (et == 0) {
-          for (int r = 0; r < CS; ++r) ptx::mbar_arrive_remote(ptx::mapa_shared(xfree_bar, r));
-        }
+        release_scratch(c, et);
+        if (et == 0) { __threadfence_block(); ms->units_done = nreal + 1; }
         __syncwarp();
         if (lane == 0) ptx::mbar_arrive(&ms->unit_done);
-        ++ngemm; ++nxch; ++nreal;
+        ++ngemm; ++nx; ++nreal;
       }
     }
-    if (tr) tr[3] = ptx::globaltimer_ns();
+    if (tr) tr[5] = ptx::globaltimer_ns();
   });
   if (!ok && lane == 0) fail(c);
 }
@@ -968,7 +1052,7 @@ __global__ void __launch_bounds__(THREADS, 1) adit_loop_kernel(const __grid_cons
     ptx::mbar_init(&ms->acc_full, 1);
     ptx::mbar_init(&ms->unit_done, 4);
     ptx::mbar_init(&ms->level_go, 1);
-    ptx::mbar_init(&ms->xfull, 1);
+    ptx::mbar_init(&ms->xfull, CS * 4);
     ptx::mbar_init(&ms->xfree, CS);
     for (int s = 0; s < 2; ++s) {
       ptx::mbar_init(&ms->k_full[s], 1); ptx::mbar_init(&ms->k_empty[s], 1);
@@ -977,10 +1061,10 @@ __global__ void __launch_bounds__(THREADS, 1) adit_loop_kernel(const __grid_cons
       ptx::mbar_init(&ms->p_full[s], 4); ptx::mbar_init(&ms->pv_done[s], 1);
     }
     ptx::mbar_init(&ms->q_full, 1);
-    ptx::mbar_init(&ms->xo_ready, CS);
-    ptx::mbar_init(&ms->xo_full, 1);
     ptx::mbar_init(&ms->epi_bar, 4);
     ms->abort = 0;
+    ms->level_seen = 0;
+    ms->units_done = 0;
     ptx::fence_mbar_init();
   }
   if (warp == 3) {
