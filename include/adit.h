@@ -213,8 +213,8 @@ int adit_uses_persistent_loop(adit_handle* h, int B, int sm_budget);
 /*
  * adit_debug_wait_limit: test aid for the bounded device-side waits of the persistent kernel (no counterpart in
  * the paper).  Sets the limit of every wait to limit_ms milliseconds (default 2000) and, with withhold_level in
- * 0..7 (embed-in, embed-out, qkv, attention, o, gate/up, down, read-out), makes block 0 withhold its first
- * completion signal of that level, so that the waits for it run out: the kernel then returns normally,
+ * 0..7 (embed-in, embed-out, qkv, attention, o, gate/up, down, read-out), makes one block withhold its
+ * completion signal of the first such level of the call, so that the waits for it run out: the kernel then returns normally,
  * adit_poll_status reports ADIT_E_TIMEOUT and the call's output is unspecified.  -1 withholds nothing.
  */
 int adit_debug_wait_limit(adit_handle* h, int limit_ms, int withhold_level);

@@ -550,10 +550,10 @@ __device__ __forceinline__ float ex2f(float x) {
 __device__ __forceinline__ uint32_t swz(int r, int ch) { return (uint32_t)(r * 128 + ((ch ^ (r & 7)) << 4)); }
 
 // One level's flag: all of this block's stores of the level are ordered before the increment.
-__device__ __forceinline__ bool publish(const Ctx& c, int type, int et, bool first_of_type, int& nsync) {
+__device__ __forceinline__ bool publish(const Ctx& c, int type, int et, bool first_piece, int& nsync) {
   if (!epi_sync(c, nsync)) return false;
   if (et == 0) {
-    if (c.p->debug_skip_level == type && c.cta == 0 && first_of_type) return true;  // test aid: a flag that never comes
+    if (c.p->debug_skip_level == type && first_piece) return true;  // test aid: a completion signal that never comes
     ptx::red_release_gpu_add(c.p->counters + type, 1u);
   }
   return true;
@@ -771,7 +771,6 @@ __device__ void role_epilogue(const Ctx& c) {
   const uint32_t tm_s = c.tmem + 256;
   int nlv = 0, nreal = 0, ngemm = 0, nx = 0, nsync = 0;
   uint32_t kv_cnt = 0;
-  uint32_t seen_types = 0;  // level types this block has published at least once
   bool ok = true;
   walk_levels(p, [&](const Lv& lv) {
     if (!ok || !participates(lv, c.cid, C)) return;
@@ -779,18 +778,17 @@ __device__ void role_epilogue(const Ctx& c) {
     ++nlv;
     unsigned long long* tr = (p.trace && et == 0) ? p.trace + ((size_t)lv.seq * c.n_cta + c.cta) * 8 : nullptr;
     if (tr) tr[0] = ptx::globaltimer_ns();
-    const bool first_of_type = !((seen_types >> lv.type) & 1u);
-    seen_types |= 1u << lv.type;
     if (lv.units == 0) {
       if (tr) { tr[1] = (unsigned long long)clock64(); tr[2] = ptx::globaltimer_ns(); }
       if (lv.type == LV_EMBED_IN) level_embed_in(c, lv, et);
       else if (!level_final(c, lv, et, nsync)) { ok = false; return; }
-      if (!publish(c, lv.type, et, first_of_type, nsync)) { ok = false; return; }
+      if (!publish(c, lv.type, et, lv.k == 0 && c.cta == 0, nsync)) { ok = false; return; }
       if (tr) { tr[3] = (unsigned long long)clock64(); tr[5] = ptx::globaltimer_ns(); }
       return;
     }
     bool first_unit_of_level = true;
     for (int u = first_unit(lv, c.cid, C); u < lv.units && ok; u += C, first_unit_of_level = false) {
+      const bool first_piece = lv.k == 0 && lv.l == 0 && u == 0 && c.rank == 0;  // (the piece the test aid withholds)
       if (lv.type == LV_ATT) {
         // ================================ attention unit ================================
         const AttUnit a = att_unit(p, u, c.rank);
@@ -956,7 +954,7 @@ __device__ void role_epilogue(const Ctx& c) {
           }
         }
         ++nx;
-        if (!publish(c, LV_ATT, et, first_of_type && first_unit_of_level, nsync)) { ok = false; break; }
+        if (!publish(c, LV_ATT, et, first_piece, nsync)) { ok = false; break; }
         release_scratch(c, et);
         if (et == 0) { __threadfence_block(); ms->units_done = nreal + 1; }
         __syncwarp();
@@ -971,7 +969,7 @@ __device__ void role_epilogue(const Ctx& c) {
           if (nx > 0 && !warp_wait(c, &ms->xfree, (uint32_t)(nx - 1) & 1u)) { ok = false; break; }
           signal_partials(c);
           release_scratch(c, et);
-          if (!publish(c, lv.type, et, first_of_type && first_unit_of_level, nsync)) { ok = false; break; }
+          if (!publish(c, lv.type, et, first_piece, nsync)) { ok = false; break; }
           ++nx;
           continue;
         }
@@ -1026,7 +1024,7 @@ __device__ void role_epilogue(const Ctx& c) {
         if (nv == 2) finalize_owned<2>(c, g, gu, n_tok_valid, lane, ew, old4, rs_lane);
         else finalize_owned<1>(c, g, gu, n_tok_valid, lane, ew, old4, rs_lane);
         if (tr && first_unit_of_level) tr[4] = ptx::globaltimer_ns();
-        if (!publish(c, lv.type, et, first_of_type && first_unit_of_level, nsync)) { ok = false; break; }
+        if (!publish(c, lv.type, et, first_piece, nsync)) { ok = false; break; }
         release_scratch(c, et);
         if (et == 0) { __threadfence_block(); ms->units_done = nreal + 1; }
         __syncwarp();
