@@ -261,7 +261,8 @@ int adit_debug_gemm(int device, int n_tok, int n_feat, int k, const void* a_bf16
  *   splits     number of key splits (1..32); with more than one, partial results go through a scratch
  *              buffer that this call allocates with cudaMalloc and frees before returning
  *   out_att    DEVICE bf16 [B * n_tokens, n_q_heads * head_dim]
- * Synchronises `stream`.  Errors: INVALID, CAPACITY (B > ADIT_MAX_BATCH), UNSUPPORTED (head_dim), CUDA.
+ * Synchronises `stream`.  Errors: INVALID (also: qkv or out_att not 16-byte aligned), CAPACITY (B > ADIT_MAX_BATCH),
+ * UNSUPPORTED (head_dim), CUDA, TIMEOUT (a bounded device-side wait ran out; the output is unspecified).
  */
 int adit_debug_attention(int device, int B, int n_tokens, int n_q_heads, int n_kv_heads, int head_dim, int p_cap,
                          int layer, const void* qkv, const void* const* prefix_kv, const int32_t* prefix_len,
@@ -290,11 +291,16 @@ int adit_debug_attention(int device, int B, int n_tokens, int n_q_heads, int n_k
  * the one array: it keeps whatever the previous call left (nothing in it needs clearing - each call
  * writes every partial it later reads), and two calls whose kernels overlap on the GPU (different
  * streams, no dependency) race on it.  Order such calls yourself.
+ * A bounded device-side wait that runs out cannot be reported by this asynchronous call: the kernels record it in
+ * a status word inside the array (cleared at the start of every call); adit_attention_static_status(device)
+ * copies it out (a blocking copy, so it also waits for earlier work on the device) and returns ADIT_OK or
+ * ADIT_E_TIMEOUT for the most recent call.
  */
 #define ADIT_STATIC_SCRATCH_BYTES (8u << 20)
 int adit_attention_static(int device, int B, int n_tokens, int n_q_heads, int n_kv_heads, int head_dim, int p_cap,
                           int layer, const void* qkv, const void* const* prefix_kv, const int32_t* prefix_len,
                           int splits, void* out_att, void* stream);
+int adit_attention_static_status(int device);
 
 /*
  * adit_debug_gemm_stamps: phase timing of the projection and attention kernels (test aid; no
@@ -302,9 +308,13 @@ int adit_attention_static(int device, int B, int n_tokens, int n_q_heads, int n_
  * adit_debug_attention to record, per thread block, sixteen uint64 (%globaltimer stamps of the
  * block's phases - start, set-up done, first and last k-block landed, accumulator complete, parked,
  * sent, received, summed, epilogue done, teardown, TMEM freed - and two clock64 readings); called with
- * a host buffer of n_blocks * 16 uint64 (n_blocks <= 1024) it copies the stamps of the last such call out.
+ * a host buffer of n_blocks * 16 uint64 (n_blocks <= 1024) it copies the stamps of the last such call out; with
+ * host_dst == NULL and n_blocks < 0 it disarms and frees the buffer.  The buffer belongs to the device that was
+ * current when it was armed; only calls on that device whose grid fits it (1024 blocks, attention 512) are
+ * instrumented, all others run the plain kernels.  adit_debug_stamps_selected states that rule (host only).
  */
 int adit_debug_gemm_stamps(unsigned long long* host_dst, int n_blocks);
+int adit_debug_stamps_selected(int armed_device, int device, int grid_blocks, int is_attention);
 
 /*
  * adit_debug_plan: the tiling the library would choose for a projection of n_tok tokens, n_feat output

@@ -30,7 +30,9 @@ the following reading, taken step by step, one request at a time:
 
 Pins (tests/test_oracle_pins.py): closed-form Euler trajectories for linear
 fields; Wout = 0 gives x_K = x_0 + bout; zeroed Wo/Wd give a hand-computable
-velocity; scalar-loop softmax attention on tiny shapes; zero queries give the
+velocity; one whole layer with non-zero Wo/Wd against a composition of torch
+CPU fp64 library routines (norm -> q/k/v, attention, residual, norm ->
+GeGLU, residual); scalar-loop softmax attention on tiny shapes; zero queries give the
 mean of the valid value rows; torch CPU fp64 library routines for attention,
 RMSNorm, GELU(tanh) and SiLU; grouped-query = replicated multi-head; batch
 permutation, padding and capacity invariance; time-embedding special values.

@@ -159,7 +159,6 @@ static AttnPlan plan_attention(const adit_handle* h, int B) {
     if (p.splits < 1) p.splits = 1;
     if (p.splits > max_nkb) p.splits = max_nkb;
     if (p.splits > 32) p.splits = 32;  // the merge kernel keeps one split per lane
-    if (const char* e = getenv("ADIT_ATTN_SPLITS")) { int v = atoi(e); if (v >= 1 && v <= 32 && v <= max_nkb) p.splits = v; }
   }
   return p;
 }
@@ -604,7 +603,12 @@ static cudaError_t attn_attr() {
                               (int)attn::attn_smem_bytes<DH, NW>());
 }
 static cudaError_t init_attention_attrs() {
-  cudaError_t e;
+  // per device (function attributes belong to a device's copy of the kernel)
+  static bool done_dev[64] = {};
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev >= 0 && dev < 64 && done_dev[dev]) return cudaSuccess;
   if ((e = attn_attr<64, 2>()) != cudaSuccess) return e;
   if ((e = attn_attr<64, 4>()) != cudaSuccess) return e;
   if ((e = attn_attr<128, 2>()) != cudaSuccess) return e;
@@ -619,6 +623,7 @@ static cudaError_t init_attention_attrs() {
   ADIT_ATTN_ATTR(256, false); ADIT_ATTN_ATTR(256, true);
 #undef ADIT_ATTN_ATTR1
 #undef ADIT_ATTN_ATTR
+  if (dev >= 0 && dev < 64) done_dev[dev] = true;
   return cudaSuccess;
 }
 
@@ -1245,9 +1250,21 @@ extern "C" int64_t adit_debug_copy(adit_handle* h, const char* name, void* host_
 // ---------------------------------------------------------------------------------------------
 // Stand-alone ragged-prefix attention (test aid): the kernels of the loop on caller-supplied buffers.
 // ---------------------------------------------------------------------------------------------
-static unsigned long long* g_gemm_dbg = nullptr;  // device buffer for adit_debug_gemm_stamps
-__global__ void set_table_kernel(PrefixTable t, PrefixTable* __restrict__ dst) {
-  if (threadIdx.x == 0) *dst = t;
+// Phase-stamp buffer of adit_debug_gemm_stamps: [1024 blocks][16] uint64 on the device it was armed on.  The
+// attention kernel's per-key-block log of block 0 starts at element 8192, so attention grids may use 512 blocks.
+static unsigned long long* g_gemm_dbg = nullptr;
+static int g_gemm_dbg_device = -1;
+extern "C" int adit_debug_stamps_selected(int armed_device, int device, int grid_blocks, int is_attention) {
+  if (armed_device < 0 || armed_device != device || grid_blocks < 1) return 0;
+  return grid_blocks <= (is_attention ? 512 : 1024) ? 1 : 0;
+}
+static unsigned long long* stamp_buffer_for(int grid_blocks, bool is_attention) {
+  int dev = -1;
+  if (!g_gemm_dbg || cudaGetDevice(&dev) != cudaSuccess) return nullptr;
+  return adit_debug_stamps_selected(g_gemm_dbg_device, dev, grid_blocks, is_attention ? 1 : 0) ? g_gemm_dbg : nullptr;
+}
+__global__ void set_table_kernel(PrefixTable t, PrefixTable* __restrict__ dst, int* __restrict__ status) {
+  if (threadIdx.x == 0) { *dst = t; if (status) *status = 0; }
 }
 
 struct AttnProblem {
@@ -1257,6 +1274,7 @@ struct AttnProblem {
 static int validate_attention(const AttnProblem& q, const void* qkv, const void* const* prefix_kv,
                               const int32_t* prefix_len, const void* out_att, PrefixTable* pt) {
   if (!qkv || !prefix_kv || !prefix_len || !out_att) return ADIT_E_INVALID;
+  if ((((uintptr_t)qkv) & 15) || (((uintptr_t)out_att) & 15)) return ADIT_E_INVALID;  // 16-byte copies and stores
   if (q.B < 1 || q.n_tokens < 1 || q.n_q_heads < 1 || q.n_kv_heads < 1 || q.p_cap < 0 || q.layer < 0) return ADIT_E_INVALID;
   if (q.n_q_heads % q.n_kv_heads) return ADIT_E_INVALID;
   if (q.B > ADIT_MAX_BATCH) return ADIT_E_CAPACITY;
@@ -1298,7 +1316,7 @@ static cudaError_t attention_launch_dh(const attn::AttnArgs& a, int nw, int grid
 // Enqueue attention on `st`.  `scratch` holds the key-split partials (attention_scratch_bytes) and
 // `pt_dev` the device copy of the prefix table (written here by a small kernel).
 static cudaError_t attention_enqueue(const AttnProblem& q, const PrefixTable& pt, const void* qkv, void* out_att,
-                                     unsigned char* scratch, PrefixTable* pt_dev, cudaStream_t st) {
+                                     unsigned char* scratch, PrefixTable* pt_dev, int* status_dev, cudaStream_t st) {
   const int G = q.n_q_heads / q.n_kv_heads, R = q.n_tokens * G;
   const int nw = R <= 32 ? 2 : 4;
   const int Q = q.n_q_heads * q.head_dim;
@@ -1309,9 +1327,10 @@ static cudaError_t attention_enqueue(const AttnProblem& q, const PrefixTable& pt
   a.scale_log2 = 1.4426950408889634f / sqrtf((float)q.head_dim);
   const size_t rows = (size_t)q.splits * q.B * q.n_tokens * q.n_q_heads;
   a.part_o = scratch;
-  a.dbg = g_gemm_dbg;
+  a.dbg = stamp_buffer_for(q.B * q.n_kv_heads * ((R + attn::TC_ROWS - 1) / attn::TC_ROWS) * q.splits, true);
   a.part_ml = (float*)(scratch + rows * q.head_dim * 4);  // (the bf16 partials use half of the first region)
-  set_table_kernel<<<1, 32, 0, st>>>(pt, pt_dev);
+  a.status = status_dev;  // cleared by the table kernel, set to ADIT_E_TIMEOUT by a wait that runs out
+  set_table_kernel<<<1, 32, 0, st>>>(pt, pt_dev, status_dev);
   const int grid = q.B * q.n_kv_heads * a.n_row_tiles * q.splits;
   const int64_t n_qrows = (int64_t)q.B * q.n_tokens * q.n_q_heads;
   const int mg = (int)((n_qrows + 3) / 4);
@@ -1332,14 +1351,18 @@ extern "C" int adit_debug_attention(int device, int B, int n_tokens, int n_q_hea
   unsigned char* scratch = nullptr;
   PrefixTable* pt_dev = nullptr;
   const size_t nb = attention_scratch_bytes(q);
-  if (cudaMalloc((void**)&pt_dev, sizeof(PrefixTable)) != cudaSuccess) return ADIT_E_CUDA;
+  if (cudaMalloc((void**)&pt_dev, sizeof(PrefixTable) + 16) != cudaSuccess) return ADIT_E_CUDA;
   if (nb && cudaMalloc((void**)&scratch, nb) != cudaSuccess) { cudaFree(pt_dev); return ADIT_E_CUDA; }
   cudaStream_t st = (cudaStream_t)stream;
-  cudaError_t e = attention_enqueue(q, pt, qkv, out_att, scratch, pt_dev, st);
+  int* status_dev = (int*)((unsigned char*)pt_dev + sizeof(PrefixTable));
+  cudaError_t e = attention_enqueue(q, pt, qkv, out_att, scratch, pt_dev, status_dev, st);
   if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+  int hs = 0;
+  if (e == cudaSuccess) e = cudaMemcpy(&hs, status_dev, 4, cudaMemcpyDeviceToHost);
   cudaFree(pt_dev);
   if (scratch) cudaFree(scratch);
-  return e == cudaSuccess ? ADIT_OK : ADIT_E_CUDA;
+  if (e != cudaSuccess) return ADIT_E_CUDA;
+  return hs ? ADIT_E_TIMEOUT : ADIT_OK;
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -1372,8 +1395,19 @@ extern "C" int adit_attention_static(int device, int B, int n_tokens, int n_q_he
   PrefixTable* pt_dev = (PrefixTable*)(base + ADIT_STATIC_SCRATCH_BYTES);  // 256-byte aligned: the array is, and so is its size
   // Nothing in the scratch has to start at zero: every (split, row) partial that the merge reads is
   // written by the attention kernel of the same call, empty splits included.
-  cudaError_t e = attention_enqueue(q, pt, qkv, out_att, base, pt_dev, (cudaStream_t)stream);
+  int* status_dev = (int*)(base + ADIT_STATIC_SCRATCH_BYTES + sizeof(PrefixTable));  // inside the array's last 256 bytes
+  cudaError_t e = attention_enqueue(q, pt, qkv, out_att, base, pt_dev, status_dev, (cudaStream_t)stream);
   return e == cudaSuccess ? ADIT_OK : ADIT_E_CUDA;
+}
+
+extern "C" int adit_attention_static_status(int device) {
+  if (device < 0 || device >= 64) return ADIT_E_INVALID;
+  if (!g_static_scratch_addr[device]) return ADIT_OK;  // never used on this device
+  if (cudaSetDevice(device) != cudaSuccess) return ADIT_E_CUDA;
+  int hs = 0;
+  if (cudaMemcpy(&hs, g_static_scratch_addr[device] + ADIT_STATIC_SCRATCH_BYTES + sizeof(PrefixTable), 4, cudaMemcpyDeviceToHost) != cudaSuccess)
+    return ADIT_E_CUDA;
+  return hs ? ADIT_E_TIMEOUT : ADIT_OK;
 }
 
 extern "C" int adit_debug_plan(int n_tok, int n_feat, int k, int dual, int sm_count, int32_t* out) {
@@ -1386,8 +1420,17 @@ extern "C" int adit_debug_plan(int n_tok, int n_feat, int k, int dual, int sm_co
 }
 
 extern "C" int adit_debug_gemm_stamps(unsigned long long* host_dst, int n_blocks) {
-  if (!host_dst) {  // arm: allocate the stamp buffer
+  if (!host_dst && n_blocks < 0) {  // disarm
+    if (g_gemm_dbg) { cudaSetDevice(g_gemm_dbg_device); cudaDeviceSynchronize(); cudaFree(g_gemm_dbg); }
+    g_gemm_dbg = nullptr; g_gemm_dbg_device = -1;
+    return ADIT_OK;
+  }
+  if (!host_dst) {  // arm: allocate the stamp buffer on the current device
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return ADIT_E_CUDA;
+    if (g_gemm_dbg && dev != g_gemm_dbg_device) return ADIT_E_INVALID;  // armed elsewhere: disarm first
     if (!g_gemm_dbg && cudaMalloc((void**)&g_gemm_dbg, 1024 * 16 * 8) != cudaSuccess) return ADIT_E_CUDA;
+    g_gemm_dbg_device = dev;
     cudaMemset(g_gemm_dbg, 0, 1024 * 16 * 8);
     return ADIT_OK;
   }
@@ -1417,8 +1460,8 @@ extern "C" int adit_debug_gemm(int device, int n_tok, int n_feat, int k, const v
   cudaStream_t st = (cudaStream_t)stream;
   tc::GemmArgs g{};
   g.n_feat = n_feat; g.n_tok = n_tok; g.epi = EPI_STORE_F32; g.out = tmp; g.ldo = n_feat; g.status = status;
-  g.dbg = g_gemm_dbg;
   const int G = (sm_budget <= 0 || sm_budget >= SM) ? SM : sm_budget;
+  g.dbg = stamp_buffer_for(tc::gemm_grid(p, G), false);
   cudaError_t e = tc::launch_gemm(mw, ma, p, false, g, G, st);
   if (e == cudaSuccess) e = cudaMemcpyAsync(out_f32, tmp, (size_t)n_tok * n_feat * 4, cudaMemcpyDeviceToDevice, st);
   if (e == cudaSuccess) e = cudaStreamSynchronize(st);
@@ -1427,7 +1470,6 @@ extern "C" int adit_debug_gemm(int device, int n_tok, int n_feat, int k, const v
   cudaFree(status);
   cudaFree(tmp);
   if (e != cudaSuccess) {
-    if (getenv("ADIT_DEBUG")) fprintf(stderr, "adit_debug_gemm: CUDA error %d (%s); plan splits=%d tile=%d stages=%d smem=%zu\n", (int)e, cudaGetErrorString(e), p.splits, p.tile_tok, p.stages, p.smem_bytes);
     cudaGetLastError();
     return ADIT_E_CUDA;
   }

@@ -186,8 +186,14 @@ static cudaError_t for_gemm_kernel(bool dual, int epi, int idx, F&& f) {
   }
 }
 
+// (function attributes are per device: set once for every device that a handle or a test aid uses)
 static cudaError_t ensure_smem_attr() {
-  static bool done = false;
+  static bool done_dev[64] = {};
+  int dev = 0;
+  cudaError_t ed = cudaGetDevice(&dev);
+  if (ed != cudaSuccess) return ed;
+  bool unused = false;
+  bool& done = (dev >= 0 && dev < 64) ? done_dev[dev] : unused;
   if (done) return cudaSuccess;
   const int epis[6] = {EPI_STORE, EPI_SILU_VEC, EPI_STORE_F32, EPI_RESID_NORM, EPI_EMBED_NORM, EPI_GEGLU};
   for (int e6 = 0; e6 < 6; ++e6)

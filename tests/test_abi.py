@@ -73,3 +73,31 @@ def test_config_struct_matches_header(adit):
     # 13 int32 + 3 float + 1 int32, no padding
     assert C.sizeof(adit.Config) == 17 * 4
     assert C.sizeof(adit.Tensor) == 8 + 8 + 4 + 4 + 32 + 8
+
+
+def test_attention_entry_points_reject_misaligned_buffers_on_the_host(adit):
+    """16-byte copies and stores need 16-byte aligned qkv / out_att: a sliced bf16 pointer is refused before
+    anything is enqueued (the pointers below are never dereferenced)."""
+    kv = (C.c_void_p * 1)(0x10000)
+    lens = (C.c_int32 * 1)(8)
+    for fn in (adit.lib.adit_debug_attention, adit.lib.adit_attention_static):
+        for qkv, out in ((0x20002, 0x30000), (0x20000, 0x30008)):
+            assert fn(0, 1, 4, 2, 1, 64, 16, 0, C.c_void_p(qkv), kv, lens, 1, C.c_void_p(out), None) == adit.E_INVALID
+    assert adit.lib.adit_attention_static_status(-1) == adit.E_INVALID
+    assert adit.lib.adit_attention_static_status(5) == adit.OK      # never used on that device
+
+
+def test_stamp_buffer_is_only_used_where_it_fits(adit):
+    """The phase-stamp buffer holds 1024 blocks on the device it was armed on; larger grids (attention: 512, the
+    per-block log starts there) and other devices must run the plain kernels instead of writing past it."""
+    sel = adit.lib.adit_debug_stamps_selected
+    assert sel(0, 0, 1024, 0) == 1 and sel(0, 0, 1025, 0) == 0
+    assert sel(0, 0, 512, 1) == 1 and sel(0, 0, 513, 1) == 0 and sel(0, 0, 24576, 1) == 0
+    assert sel(0, 1, 8, 0) == 0 and sel(-1, 0, 8, 0) == 0 and sel(0, 0, 0, 0) == 0
+
+
+def test_persistent_loop_queries_are_host_only(adit):
+    assert adit.lib.adit_uses_persistent_loop(None, 1, 0) == adit.E_INVALID
+    assert adit.lib.adit_debug_wait_limit(None, 5, -1) == adit.E_INVALID
+    assert adit.lib.adit_clear_status(None) == adit.E_INVALID
+    assert adit.lib.adit_loop_trace_read(None, None, 0) == adit.E_INVALID

@@ -157,8 +157,16 @@ def test_slot_batch_size_budget_and_repeat_are_bit_identical(adit, dtype):
                           torch.from_numpy(wl.noise[b:b + 1]).cuda(), wl.n_steps).cpu().numpy()
         if dtype == "fp32":
             assert np.array_equal(got[0].view(np.uint32), base[b].view(np.uint32)), b
-        else:   # the k-split of the projections depends on the batch size: same value up to rounding order
-            assert np.abs(got[0] - base[b]).max() <= 3e-2, b
+        else:
+            # The k-split of the projections and the key split of the attention follow the token count, so a request
+            # alone and the same request in a batch of nine are two bf16 evaluations in different summation orders.
+            # Their gap is of the size of either one's distance to the fp64 oracle (observed here: max-abs <= 9e-3,
+            # relative L2 <= 2.5e-3); a value leaking from another request would show as a gap of the size of the
+            # values themselves (order 1).  Bound: about twice the observed gap.
+            gap = np.abs(got[0] - base[b]).max()
+            rel = np.linalg.norm(got[0] - base[b]) / np.linalg.norm(base[b])
+            print("alone vs in batch", b, gap, rel)
+            assert gap <= 2e-2 and rel <= 5e-3, (b, gap, rel)
     # output may alias the noise buffer
     nz = torch.from_numpy(wl.noise).cuda()
     eng.denoise(kv, wl.prefix_len, torch.from_numpy(wl.state).cuda(), nz, wl.n_steps, out=nz)
@@ -190,6 +198,43 @@ def test_prefix_rows_do_matter(adit):
     for b in range(wl.batch):
         same = np.array_equal(got[b].view(np.uint32), base[b].view(np.uint32))
         assert same == (b not in (2, 8)), b
+
+
+def test_two_experts_on_two_streams_at_once(adit):
+    """Two handles of different shape families enqueued on two streams before either is synchronised (the
+    co-located experts of the paper's section 4.1.3): both results against the oracle, and bitwise equal to each
+    expert running alone."""
+    import torch
+    cases = []
+    for name, cfg, plens, cap, steps, flags in (
+            ("pi0", W.scaled(W.PI0, n_layers=2), [130, 0, 257, 64], 320, 3, 0),
+            ("expert2", W.scaled(W.EXPERT2, n_layers=2), [256, 31, 64, 1, 100], 256, 2, 0),
+            ("pi0-persistent", W.scaled(W.PI0, n_layers=2), [77], 128, 2, adit.FLAG_PERSISTENT_LOOP),
+            ("tiny-persistent", W.scaled(W.TINY, dtype="bf16"), [64, 5], 96, 3, adit.FLAG_PERSISTENT_LOOP)):
+        wl = W.make_workload(name, cfg, seed=51, batch=len(plens), n_steps=steps, prefix_len=plens, max_prefix_len=cap)
+        w = W.make_weights(cfg, wl.seed)
+        eng = adit.ADiT(cfg, max_batch=len(plens), max_prefix_len=cap, flags=flags)
+        eng.load_weights(w)
+        cases.append({"wl": wl, "w": w, "eng": eng, "kv": adit.upload_prefix_kv(wl), "stream": torch.cuda.Stream(),
+                      "state": torch.from_numpy(wl.state).cuda(), "noise": torch.from_numpy(wl.noise).cuda()})
+    alone = []
+    for c in cases:
+        alone.append(c["eng"].denoise(c["kv"], c["wl"].prefix_len, c["state"], c["noise"], c["wl"].n_steps).cpu().numpy())
+    torch.cuda.synchronize()
+    for _ in range(2):
+        outs = []
+        for rep in range(3):                       # several calls per stream in flight, nothing synchronised in between
+            for c in cases:
+                outs.append(c["eng"].denoise(c["kv"], c["wl"].prefix_len, c["state"], c["noise"], c["wl"].n_steps,
+                                             stream=c["stream"]))
+        torch.cuda.synchronize()
+        for i, o in enumerate(outs):
+            c = cases[i % len(cases)]
+            assert c["eng"].poll_status() == 0
+            assert np.array_equal(o.cpu().numpy().view(np.uint32), alone[i % len(cases)].view(np.uint32)), c["wl"].name
+    for c, a in zip(cases, alone):
+        check(a, oracle(c["wl"], c["w"]), "bf16", c["wl"].name)
+        c["eng"].close()
 
 
 # ---- errors reported through status codes -------------------------------------------------------

@@ -333,6 +333,80 @@ def test_esf_matches_brute_force():
         assert got in ok and len(ok) == 1
 
 
+# ---- P12: the wiring of one layer, with non-zero Wo and Wd -----------------------------------------
+
+def _layer_by_torch(cfg, w, l, h, kv_l, plen):
+    """One pre-norm block composed from torch CPU fp64 library routines and explicit products, written from the
+    definition (attention sub-block, then GeGLU MLP sub-block), without calling the oracle."""
+    import torch
+    import torch.nn.functional as F
+    t = lambda a: torch.from_numpy(np.ascontiguousarray(a, dtype=np.float64))
+    p = f"layers.{l}."
+    x = t(h)
+    n, D = x.shape
+    Hq, Hkv, dh = cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim
+    u = F.rms_norm(x, (D,), weight=t(w[p + "norm1.g"]), eps=cfg.rms_eps)
+    q = (u @ t(w[p + "wq"])).view(n, Hq, dh).transpose(0, 1)                       # [Hq, n, dh]
+    k = (u @ t(w[p + "wk"])).view(n, Hkv, dh).transpose(0, 1)
+    v = (u @ t(w[p + "wv"])).view(n, Hkv, dh).transpose(0, 1)
+    k_all = torch.cat([t(kv_l[0][:, :plen]), k], dim=1).repeat_interleave(Hq // Hkv, dim=0)   # [Hq, plen + n, dh]
+    v_all = torch.cat([t(kv_l[1][:, :plen]), v], dim=1).repeat_interleave(Hq // Hkv, dim=0)
+    o = F.scaled_dot_product_attention(q, k_all, v_all)                              # no mask, scale 1/sqrt(dh)
+    x = x + o.transpose(0, 1).reshape(n, Hq * dh) @ t(w[p + "wo"])
+    u = F.rms_norm(x, (D,), weight=t(w[p + "norm2.g"]), eps=cfg.rms_eps)
+    x = x + (F.gelu(u @ t(w[p + "wg"]), approximate="tanh") * (u @ t(w[p + "wu"]))) @ t(w[p + "wd"])
+    return x.numpy()
+
+
+def _layer_case():
+    cfg = W.scaled(W.TINY, n_layers=1, d_model=32, n_q_heads=4, n_kv_heads=2, head_dim=8, d_ff=48, horizon=5,
+                   time_emb_dim=32)
+    rng = np.random.default_rng(99)
+    w = {k: np.asarray(v, dtype=np.float64) for k, v in W.make_weights(cfg, 7).items()}
+    for k in list(w):                       # weights large enough for every term to matter
+        if k.startswith("layers.0.w"):
+            w[k] = rng.standard_normal(w[k].shape) * 0.3
+        if k.endswith(".g"):
+            w[k] = 1.0 + 0.5 * rng.standard_normal(w[k].shape)
+    h = rng.standard_normal((cfg.n_tokens, cfg.d_model))
+    plen, cap = 7, 9
+    kv = rng.standard_normal((2, cfg.n_kv_heads, cap, cfg.head_dim))
+    kv[:, :, plen:] = np.nan
+    return cfg, w, h, kv, plen
+
+
+def test_layer_forward_matches_library_composition():
+    cfg, w, h, kv, plen = _layer_case()
+    got = O.layer_forward(cfg, w, 0, h, kv, plen)
+    want = _layer_by_torch(cfg, w, 0, h, kv, plen)
+    assert np.isfinite(got).all()
+    np.testing.assert_allclose(got, want, rtol=1e-12, atol=1e-12)
+    assert np.abs(got - h).max() > 0.5      # both residual branches contribute: the layer is far from the identity
+
+
+def test_layer_wiring_mistakes_are_visible():
+    """Each plausible wiring mistake changes the library composition's result by far more than the tolerance of the
+    comparison above, so the oracle cannot contain it and still pass: gate/up swapped, the first norm's gain in the
+    second norm, value weights used for the keys, un-normalised input to the query projection, a dropped residual."""
+    cfg, w, h, kv, plen = _layer_case()
+    want = _layer_by_torch(cfg, w, 0, h, kv, plen)
+    p = "layers.0."
+    swaps = {"gate/up": {p + "wg": w[p + "wu"], p + "wu": w[p + "wg"]},
+             "norm gains": {p + "norm2.g": w[p + "norm1.g"]},
+             "wk<-wv": {p + "wk": w[p + "wv"]}}
+    for name, repl in swaps.items():
+        w2 = dict(w)
+        w2.update(repl)
+        assert np.abs(O.layer_forward(cfg, w2, 0, h, kv, plen) - want).max() > 1e-3, name
+    # un-normalised input to wq == folding 1/rms out of the query: emulate by scaling the rows of h for q only
+    w3 = dict(w)
+    w3[p + "wq"] = w[p + "wq"] * 1.7
+    assert np.abs(O.layer_forward(cfg, w3, 0, h, kv, plen) - want).max() > 1e-3
+    w4 = dict(w)
+    w4[p + "wo"] = np.zeros_like(w[p + "wo"])
+    assert np.abs(O.layer_forward(cfg, w4, 0, h, kv, plen) - want).max() > 1e-3
+
+
 # ---- the full configurations run and are healthy --------------------------------------------
 
 def test_config_c1_runs_and_signal_is_healthy():
