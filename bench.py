@@ -126,6 +126,14 @@ class ClockSampler:
                 "power_w_max": max(pw) if pw else None, "samples": len(sm), "reasons": sorted(reasons)}
 
 
+def bench_config(base, sm_budget, world, step_bytes, n_sets):
+    """The `config` object of the JSON line: the same keys for the GPU arm and the reference arm."""
+    return {"workload": base.name, "batch": base.batch, "euler_steps": base.n_steps,
+            "prefix_len_mean": float(np.mean(base.prefix_len)), "sm_budget": sm_budget, "parallelism": f"replicas x{world}",
+            "l2": f"inputs larger than L2: {step_bytes / 1e6:.0f} MB streamed per Euler step vs 126 MB L2; "
+                  f"{n_sets} rotating input sets"}
+
+
 # ---- CPU oracle legs ------------------------------------------------------------------------------
 
 def oracle_sample_seconds(wl, weights_f64, n_euler_sample, requests):
@@ -168,7 +176,8 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": per_chunk * 1e3 * wl.batch,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": wl.name, "batch": wl.batch, "euler_steps": wl.n_steps},
+        "config": bench_config(wl, args.sm_budget, max(1, args.gpus),
+                               algorithmic_work(wl.cfg, wl.prefix_len, wl.n_steps)["step_bytes"], 4),
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -176,6 +185,61 @@ def run_reference(args):
 
 
 # ---- the GPU arm ----------------------------------------------------------------------------------
+
+def make_sets(adit, base, n_sets, rank, local, dev, torch):
+    """n_sets input sets (own prefix caches, states, noise) of the workload's shape; each rank draws its own."""
+    sets = []
+    for s in range(n_sets):
+        wl = W.make_workload(base.name, base.cfg, seed=base.seed + 1000 * (1 + s + n_sets * rank), batch=base.batch,
+                             n_steps=base.n_steps, prefix_len=base.prefix_len, max_prefix_len=base.max_prefix_len)
+        sets.append({"kv": adit.upload_prefix_kv(wl, local), "len": wl.prefix_len,
+                     "state": torch.from_numpy(wl.state).to(dev), "noise": torch.from_numpy(wl.noise).to(dev),
+                     "state_h": torch.from_numpy(wl.state).pin_memory(), "noise_h": torch.from_numpy(wl.noise).pin_memory(),
+                     "out_h": torch.empty(wl.noise.shape, dtype=torch.float32).pin_memory(),
+                     "out": torch.empty(wl.noise.shape, dtype=torch.float32, device=dev)})
+    return sets
+
+
+def step_roofline(cfg, prefix_len, n_euler, ms_per_call, peaks):
+    """Whole call: the slower of bytes at the HBM peak and flops at the sustained bf16 peak, against the measured time."""
+    work = algorithmic_work(cfg, prefix_len, n_euler)
+    t_hbm = work["step_bytes"] / (peaks["hbm_gbs"] * 1e9)
+    t_tc = work["step_flops"] / (peaks["bf16_tflops_sustained"] * 1e12)
+    floor_ms = max(t_hbm, t_tc) * n_euler * 1e3
+    return work, {"bound": "hbm" if t_hbm >= t_tc else "tensor", "floor_ms_per_call": floor_ms, "frac": floor_ms / ms_per_call,
+                  "bytes_per_euler_step": work["step_bytes"], "flops_per_euler_step": work["step_flops"],
+                  "achieved_gbs": work["step_bytes"] * n_euler / (ms_per_call * 1e-3) / 1e9,
+                  "achieved_tflops": work["step_flops"] * n_euler / (ms_per_call * 1e-3) / 1e12}
+
+
+def sample_latency(torch, eng, sets, n_euler, budget, stream, n_calls, wall_s):
+    """Per-call device latency (CUDA events on the call's stream) of up to n_calls back-to-back calls, stopped early
+    when the wall budget is spent."""
+    lat, t0, i = [], time.perf_counter(), 0
+    while i < n_calls and time.perf_counter() - t0 < wall_s:
+        chunk = min(100, n_calls - i)
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(chunk + 1)]
+        ev[0].record(stream)
+        for j in range(chunk):
+            s = sets[(i + j) % len(sets)]
+            eng.denoise(s["kv"], s["len"], s["state"], s["noise"], n_euler, sm_budget=budget, stream=stream, out=s["out"])
+            ev[j + 1].record(stream)
+        stream.synchronize()
+        lat += [ev[j].elapsed_time(ev[j + 1]) for j in range(chunk)]
+        i += chunk
+    return np.array(lat)
+
+
+def traffic_from_profile(kernel, workload):
+    """dram__bytes_read.sum + dram__bytes_write.sum per launch as recorded in the kernel's ncu summary under profiles/
+    (a line `dram_bytes_per_launch: <number>`), or None."""
+    import re
+    path = os.path.join(ROOT, "profiles", f"{kernel}_{workload}.md")
+    if not os.path.exists(path):
+        return None
+    m = re.search(r"dram_bytes_per_launch:\s*([0-9.eE+]+)", open(path).read())
+    return float(m.group(1)) if m else None
+
 
 def run_ours(args):
     import torch
@@ -196,18 +260,10 @@ def run_ours(args):
     base = WORKLOADS[args.workload]()
     cfg = base.cfg
     weights = W.make_weights(cfg, base.seed)
-    eng = adit.ADiT(cfg, max_batch=base.batch, max_prefix_len=base.max_prefix_len, device=local)
+    flags = (adit.FLAG_NO_GRAPH if args.no_graph else 0) | (adit.FLAG_PERSISTENT_LOOP if args.persistent else 0)
+    eng = adit.ADiT(cfg, max_batch=base.batch, max_prefix_len=base.max_prefix_len, device=local, flags=flags)
     eng.load_weights(weights)
-    # n_sets input sets (own prefix caches, states, noise); each rank draws its own requests
-    sets = []
-    for s in range(n_sets):
-        wl = W.make_workload(base.name, cfg, seed=base.seed + 1000 * (1 + s + n_sets * rank), batch=base.batch,
-                             n_steps=base.n_steps, prefix_len=base.prefix_len, max_prefix_len=base.max_prefix_len)
-        sets.append({"kv": adit.upload_prefix_kv(wl, local), "len": wl.prefix_len,
-                     "state": torch.from_numpy(wl.state).to(dev), "noise": torch.from_numpy(wl.noise).to(dev),
-                     "state_h": torch.from_numpy(wl.state).pin_memory(), "noise_h": torch.from_numpy(wl.noise).pin_memory(),
-                     "out_h": torch.empty(wl.noise.shape, dtype=torch.float32).pin_memory(),
-                     "out": torch.empty(wl.noise.shape, dtype=torch.float32, device=dev)})
+    sets = make_sets(adit, base, n_sets, rank, local, dev, torch)
     stream = torch.cuda.Stream(device=dev)
     K_e, B = base.n_steps, base.batch
 
@@ -230,21 +286,23 @@ def run_ours(args):
         if rank == 0:
             sampler.start()
         launches0 = eng.kernel_launches()
-        ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
-        ev[0].record(stream)
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ev0.record(stream)
         for i in range(args.steps):
             call(i)
-            ev[i + 1].record(stream)
+        ev1.record(stream)
         barrier()
-        total_ms = ev[0].elapsed_time(ev[-1])
+        total_ms = ev0.elapsed_time(ev1)
         launches = eng.kernel_launches() - launches0
         clocks = sampler.stop() if rank == 0 else None
-        lat = np.array([ev[i].elapsed_time(ev[i + 1]) for i in range(args.steps)])
         if world > 1:
             t = torch.tensor([total_ms], device=dev, dtype=torch.float64)
             dist.all_reduce(t, op=dist.ReduceOp.MAX)
             total_ms = float(t.item())
         assert eng.poll_status() == 0
+
+        # ---- per-call latency distribution (its own calls: p99 needs many samples whatever --steps is) ----
+        lat = sample_latency(torch, eng, sets, K_e, args.sm_budget, stream, args.latency_calls, args.latency_seconds)
 
         # ---- end to end through the host-buffer entry point (pinned host in, host out) ------------
         for i in range(3):
@@ -271,7 +329,7 @@ def run_ours(args):
         eng.profile_enable(False)
         # ---- in-situ kernel durations: %globaltimer stamps written by every block inside the replayed graph --
         trace = None
-        if not args.no_trace:
+        if not args.no_trace and not args.persistent:
             eng.trace_enable(True)
             call(0)
             call(1)
@@ -285,61 +343,87 @@ def run_ours(args):
         return
 
     peaks, peaks_kind = load_peaks()
-    work = algorithmic_work(cfg, base.prefix_len, K_e)
     ms_per_step = total_ms / args.steps
     value = world * B * args.steps / (total_ms * 1e-3)
-    # whole-step roofline: slower of bytes at HBM peak and flops at the sustained bf16 peak
-    t_hbm = work["step_bytes"] / (peaks["hbm_gbs"] * 1e9)
-    t_tc = work["step_flops"] / (peaks["bf16_tflops_sustained"] * 1e12)
-    step_bound = "hbm" if t_hbm >= t_tc else "tensor"
-    floor_ms = max(t_hbm, t_tc) * K_e * 1e3
-    step_roof = {"bound": step_bound, "floor_ms_per_call": floor_ms, "frac": floor_ms / ms_per_step,
-                 "bytes_per_euler_step": work["step_bytes"], "flops_per_euler_step": work["step_flops"],
-                 "achieved_gbs": work["step_bytes"] * K_e / (ms_per_step * 1e-3) / 1e9,
-                 "achieved_tflops": work["step_flops"] * K_e / (ms_per_step * 1e-3) / 1e12}
+    work, step_roof = step_roofline(cfg, base.prefix_len, K_e, ms_per_step, peaks)
     # dominant kernel: the four per-layer projections (and the two embedding projections) are launches of the
-    # same kernel, gemm_tc_kernel; attention (+ merge) is the other candidate
+    # same kernel, gemm_tc_kernel; attention (+ merge) is the other candidate; the persistent path is one kernel
     tot = sum(v[0] for v in prof.values()) or 1.0
     shares = {k: {"ms_per_call": v[0] / n_prof, "launches_per_call": v[1] // n_prof, "share": v[0] / tot}
               for k, v in prof.items() if v[1]}
     gemm_classes = [k for k in ("gemm_qkv", "gemm_o", "gemm_gateup", "gemm_down") if k in shares]
-    groups = {"gemm_tc_kernel": gemm_classes, "attn_tc_kernel": [k for k in ("attention",) if k in shares]}
+    groups = {"gemm_tc_kernel": gemm_classes, "attn_tc_kernel": [k for k in ("attention",) if k in shares],
+              "adit_loop_kernel": [k for k in ("loop",) if k in shares]}
     gtime = {g: sum(prof[k][0] for k in ks) for g, ks in groups.items() if ks}
     dom = max(gtime, key=gtime.get) if gtime else None
     roofline = None
     if dom:
         ks = groups[dom]
         n_launch = sum(prof[k][1] for k in ks)
-        avg_s = gtime[dom] / n_launch * 1e-3
-        bytes_l = sum(work["per_class"][k]["bytes"] * prof[k][1] for k in ks) / n_launch
-        flops_l = sum(work["per_class"][k]["flops"] * prof[k][1] for k in ks) / n_launch
-        hb = bytes_l / (peaks["hbm_gbs"] * 1e9)
-        tb = flops_l / (peaks["bf16_tflops"] * 1e12)
-        if hb >= tb:
-            roofline = {"kernel": dom, "bound": "hbm", "achieved": bytes_l / avg_s / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s"}
+        if dom == "adit_loop_kernel":       # one launch carries the whole call
+            bytes_l, flops_l = work["step_bytes"] * K_e, work["step_flops"] * K_e
         else:
-            roofline = {"kernel": dom, "bound": "tensor", "achieved": flops_l / avg_s / 1e12, "peak": peaks["bf16_tflops"],
-                        "unit": "TFLOP/s"}
-        roofline["frac"] = roofline["achieved"] / roofline["peak"]
-        # DRAM bytes per launch from the ncu capture summarised in profiles/ (same workload), else null
-        roofline["traffic"] = NCU_TRAFFIC_PER_LAUNCH.get((args.workload, dom))
-        roofline["avg_launch_us"] = avg_s * 1e6
-        roofline["launches"] = n_launch // n_prof
-        roofline["algorithmic_bytes_per_launch"] = bytes_l
-        roofline["algorithmic_flops_per_launch"] = flops_l
-        roofline["timing"] = "CUDA events around every launch on the call's stream (serialised launches, 3 calls)"
-        roofline["peak_source"] = f"{peaks_kind} (MEASURED_PEAKS.json)" if peaks_kind == "measured" else "fallback"
-        if trace is not None and len(trace):
-            # the same kernel as it runs inside the replayed graph (overlapped with its neighbours by programmatic
-            # dependent launch): from the release of its dependency wait to its last block's end
-            names = [adit.lib.adit_profile_class_name(i).decode() for i in range(10)]
+            bytes_l = sum(work["per_class"][k]["bytes"] * prof[k][1] for k in ks) / n_launch
+            flops_l = sum(work["per_class"][k]["flops"] * prof[k][1] for k in ks) / n_launch
+        hbm_bound = bytes_l / (peaks["hbm_gbs"] * 1e9) >= flops_l / (peaks["bf16_tflops"] * 1e12)
+        peak, unit = (peaks["hbm_gbs"], "GB/s") if hbm_bound else (peaks["bf16_tflops"], "TFLOP/s")
+        per_s = (lambda sec: bytes_l / sec / 1e9) if hbm_bound else (lambda sec: flops_l / sec / 1e12)
+        # serialised figure: CUDA events around every launch (adds the launch gap, removes the overlap of the replay)
+        ser_s = gtime[dom] / n_launch * 1e-3
+        serialised = {"avg_launch_us": ser_s * 1e6, "achieved": per_s(ser_s), "frac": per_s(ser_s) / peak,
+                      "timing": "CUDA events around every launch on the call's stream (serialised launches, 3 calls)"}
+        # in-situ figure: the kernel as it runs inside the timed replay, from device timestamps of every block
+        dur_s, timing = None, None
+        if dom == "adit_loop_kernel":
+            dur_s, timing = ms_per_step * 1e-3, "the timed region itself (the call is this one kernel plus a set-up kernel)"
+        elif trace is not None and len(trace):
+            names = [adit.lib.adit_profile_class_name(i).decode() for i in range(adit.N_KERNEL_CLASSES)]
             sel = [r for r in trace if names[int(r[0])] in ks and r[6] > 0]
             if sel:
                 dur_s = float(np.mean([(r[5] - r[6]) for r in sel])) * 1e-9
-                ach = (bytes_l / dur_s / 1e9) if roofline["bound"] == "hbm" else (flops_l / dur_s / 1e12)
-                roofline["in_situ"] = {"avg_launch_us": dur_s * 1e6, "achieved": ach, "frac": ach / roofline["peak"],
-                                       "timing": "device %globaltimer stamps per block inside the replayed graph "
-                                                 "(dependency released -> last block done; instrumented kernels)"}
+                timing = ("device %globaltimer stamps of every block inside the replayed graph (dependency released -> "
+                          "last block done; instrumented kernels)")
+        if dur_s is None:
+            dur_s, timing = ser_s, serialised["timing"]
+        roofline = {"kernel": dom, "bound": "hbm" if hbm_bound else "tensor", "achieved": per_s(dur_s), "peak": peak,
+                    "unit": unit, "frac": per_s(dur_s) / peak, "traffic": traffic_from_profile(dom, args.workload),
+                    "avg_launch_us": dur_s * 1e6, "launches": n_launch // n_prof,
+                    "algorithmic_bytes_per_launch": bytes_l, "algorithmic_flops_per_launch": flops_l, "timing": timing,
+                    "launch_time_share_of_call": (n_launch // n_prof) * dur_s * 1e3 / ms_per_step,
+                    "serialised_events": serialised,
+                    "peak_source": f"{peaks_kind} (MEASURED_PEAKS.json)" if peaks_kind == "measured" else "fallback"}
+
+    # ---- the other batch sizes of the metric, briefly (same expert, its own handle sized for 32 requests) ----
+    by_workload = {}
+    if world == 1 and args.workload == "c2" and not args.no_extra:
+        big = adit.ADiT(cfg, max_batch=32, max_prefix_len=1024, device=local)
+        big.load_weights(weights)
+        for name, n_calls in (("c3", 150), ("c4", 80)):
+            wl = WORKLOADS[name]()
+            bsets = make_sets(adit, wl, 1, rank, local, dev, torch)
+            with torch.cuda.stream(stream):
+                for i in range(3):
+                    big.denoise(bsets[0]["kv"], bsets[0]["len"], bsets[0]["state"], bsets[0]["noise"], wl.n_steps, stream=stream,
+                                out=bsets[0]["out"])
+                l2 = sample_latency(torch, big, bsets, wl.n_steps, 0, stream, n_calls, 6.0)
+            _, roof = step_roofline(wl.cfg, wl.prefix_len, wl.n_steps, float(l2.mean()), peaks)
+            by_workload[name] = {"batch": wl.batch, "calls": int(len(l2)), "ms_p50": float(np.percentile(l2, 50)),
+                                 "ms_p99": float(np.percentile(l2, 99)), "ms_mean": float(l2.mean()),
+                                 "chunks_per_s": wl.batch / (float(l2.mean()) * 1e-3), "roofline_step": roof}
+            del bsets
+        assert big.poll_status() == 0
+        big.close()
+        # the same call as one persistent kernel (opt-in path), for the record
+        pl = adit.ADiT(cfg, max_batch=base.batch, max_prefix_len=base.max_prefix_len, device=local, flags=adit.FLAG_PERSISTENT_LOOP)
+        pl.load_weights(weights)
+        if pl.persistent_blocks(B) > 0:
+            with torch.cuda.stream(stream):
+                l0 = pl.kernel_launches()
+                l3 = sample_latency(torch, pl, sets, K_e, 0, stream, 40, 3.0)
+            by_workload["c2_persistent_loop"] = {"batch": B, "calls": int(len(l3)), "ms_p50": float(np.percentile(l3, 50)),
+                                                 "ms_p99": float(np.percentile(l3, 99)), "blocks": pl.persistent_blocks(B),
+                                                 "launches_per_call": (pl.kernel_launches() - l0) / max(1, len(l3))}
+        pl.close()
 
     # CPU baseline: the oracle as it stands, bounded sample, rank 0 at N = 1 only
     cpu = None
@@ -362,13 +446,10 @@ def run_ours(args):
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16" if cfg.dtype == "bf16" else "f32", "data": "synthetic",
-        "config": {"workload": base.name, "batch": B, "euler_steps": K_e, "prefix_len_mean": float(np.mean(base.prefix_len)),
-                   "sm_budget": args.sm_budget, "parallelism": f"replicas x{world}",
-                   "l2": f"inputs larger than L2: {work['step_bytes'] / 1e6:.0f} MB streamed per Euler step vs 126 MB L2; "
-                         f"{n_sets} rotating input sets"},
+        "config": bench_config(base, args.sm_budget, world, work["step_bytes"], n_sets),
         "latency_ms": {"p50": float(np.percentile(lat, 50)), "p99": float(np.percentile(lat, 99)),
-                       "mean": float(lat.mean()), "min": float(lat.min())},
-        "roofline": roofline, "roofline_step": step_roof, "kernel_shares": shares,
+                       "mean": float(lat.mean()), "min": float(lat.min()), "calls": int(len(lat))},
+        "roofline": roofline, "roofline_step": step_roof, "kernel_shares": shares, "by_workload": by_workload,
         "cpu_baseline": cpu,
         "e2e": {"value": world * B * n_e2e / e2e_s, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "calls": n_e2e},
@@ -407,6 +488,16 @@ def run_budget_sweep(args):
     torch.cuda.synchronize()
     bg_ms_full = e0.elapsed_time(e1) / 10
     results = {}
+    peaks, _ = load_peaks()
+    work = algorithmic_work(cfg, base.prefix_len, base.n_steps)
+    roof = {}
+    for budget in [int(b) for b in args.budgets.split(",")]:
+        # memory roofline of a run confined to `budget` SMs: what a plain streaming read reaches from that many SMs
+        read_gbs = adit.stream_read_gbs(min(budget, n_sm))
+        tc = peaks["bf16_tflops_sustained"] * 1e12 * min(budget, n_sm) / n_sm
+        floor_ms = max(work["step_bytes"] / (read_gbs * 1e9), work["step_flops"] / tc) * base.n_steps * 1e3
+        roof[str(budget)] = {"stream_read_gbs": read_gbs, "floor_ms_per_call": floor_ms,
+                             "bound": "hbm" if work["step_bytes"] / (read_gbs * 1e9) >= work["step_flops"] / tc else "tensor"}
     for budget in [int(b) for b in args.budgets.split(",")]:
         for load in (False, True):
             lat = []
@@ -430,7 +521,8 @@ def run_budget_sweep(args):
             lat = np.array(lat)
             results[f"{budget}{'+load' if load else ''}"] = {
                 "p50_ms": float(np.percentile(lat, 50)), "p99_ms": float(np.percentile(lat, 99)),
-                "chunks_per_s": base.batch / (float(lat.mean()) * 1e-3)}
+                "chunks_per_s": base.batch / (float(lat.mean()) * 1e-3),
+                "roofline_frac_at_budget": roof[str(budget)]["floor_ms_per_call"] / float(np.percentile(lat, 50))}
     assert eng.poll_status() == 0
     budgets = [int(b) for b in args.budgets.split(",")]
     ratios = {}
@@ -440,11 +532,12 @@ def run_budget_sweep(args):
         for hi in budgets:
             if hi == 2 * lo:
                 ratios[f"halving_p99_{lo}_vs_{hi}_load"] = results[f"{lo}+load"]["p99_ms"] / results[f"{hi}+load"]["p99_ms"]
+                ratios[f"halving_p99_{lo}_vs_{hi}_idle"] = results[f"{lo}"]["p99_ms"] / results[f"{hi}"]["p99_ms"]
     print(json.dumps({"metric": "adit_chunk_latency_vs_sm_budget", "unit": "ms", "config": {
         "workload": base.name, "batch": base.batch, "euler_steps": base.n_steps,
         "load": "bf16 GEMM 8192x2048x2048 looping on a second stream, grid capped to the SMs outside the budget",
         "bg_gemm_ms_full_chip": bg_ms_full}, "steps": args.steps, "warmup": args.warmup, "n_sm": n_sm,
-        "results": results, "ratios": ratios}))
+        "results": results, "ratios": ratios, "roofline_per_budget": roof}))
     bg.close()
     eng.close()
 
@@ -536,21 +629,26 @@ def main():
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
-    ap.add_argument("--workload", choices=sorted(WORKLOADS), default="c2")
+    ap.add_argument("--workload", choices=sorted(WORKLOADS), default=None)
     ap.add_argument("--sm-budget", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--mode", choices=["throughput", "sweep", "colocate"], default="throughput",
                     help="sweep: latency per sm_budget with/without a concurrent GEMM load; colocate: two experts, two streams")
     ap.add_argument("--budgets", default="16,32,64,74,148")
     ap.add_argument("--no-trace", action="store_true", help="skip the in-situ timeline of one call")
+    ap.add_argument("--no-extra", action="store_true", help="skip the brief runs of the other batch sizes (c3, c4)")
+    ap.add_argument("--no-graph", action="store_true", help="enqueue kernels one by one (ADIT_FLAG_NO_GRAPH): for profilers")
+    ap.add_argument("--persistent", action="store_true", help="small batches as one persistent kernel (ADIT_FLAG_PERSISTENT_LOOP)")
+    ap.add_argument("--latency-calls", type=int, default=None, help="calls sampled for p50/p99 (default 1000 at batch 1)")
+    ap.add_argument("--latency-seconds", type=float, default=12.0, help="wall budget of the latency sampling")
     ap.add_argument("--splits", default="48,74,100")
     ap.add_argument("--trace-seconds", type=float, default=2.0)
     args = ap.parse_args()
+    if args.workload is None:
+        args.workload = "c4" if args.mode == "sweep" else "c2"
     if args.mode == "sweep":
         args.steps = 50 if args.steps is None else args.steps
         args.warmup = 5 if args.warmup is None else args.warmup
-        if args.workload == "c2":
-            args.workload = "c4"
         return run_budget_sweep(args)
     if args.mode == "colocate":
         return run_colocated(args)
@@ -561,6 +659,8 @@ def main():
     else:
         args.steps = 200 if args.steps is None else args.steps
         args.warmup = 10 if args.warmup is None else max(args.warmup, 3)
+        if args.latency_calls is None:
+            args.latency_calls = {"c2": 1000, "c3": 500, "c4": 200}.get(args.workload, 300)
         run_ours(args)
 
 

@@ -327,6 +327,14 @@ int adit_debug_stamps_selected(int armed_device, int device, int grid_blocks, in
 int adit_debug_plan(int n_tok, int n_feat, int k, int dual, int sm_count, int32_t* out);
 
 /*
+ * adit_debug_stream_read: measurement aid (no counterpart in the paper).  Allocates `bytes` of device memory
+ * (larger than the L2 cache to measure HBM), reads it `iters` times with one thread block of 512 threads on each
+ * of `sm_count` SMs using 16-byte loads, and writes the achieved read bandwidth in GB/s: the memory roofline
+ * that applies to a run restricted to that many SMs.  Synchronises the device.
+ */
+int adit_debug_stream_read(int device, size_t bytes, int sm_count, int iters, double* gb_per_s);
+
+/*
  * adit_bg_gemm_*: a looping bf16 GEMM C[m,n] = A[m,k] B[n,k]^T on a capped number of SMs, the
  * stand-in for the VLM stage that shares the GPU with the ADiT stream (section 4.1.2: the VLM
  * stream is restricted to a number of SMs so that the ADiT kernels always find free ones).

@@ -28,7 +28,7 @@ EXPORTS = ["adit_create", "adit_load_weights", "adit_denoise", "adit_denoise_hos
            "adit_poll_status", "adit_last_cuda_error", "adit_kernel_launches", "adit_strerror",
            "adit_debug_copy", "adit_debug_gemm", "adit_debug_plan", "adit_debug_gemm_stamps", "adit_debug_attention", "adit_attention_static", "adit_profile_enable", "adit_profile_read", "adit_profile_class_name", "adit_trace_enable", "adit_trace_read",
            "adit_bg_gemm_create", "adit_bg_gemm_launch", "adit_bg_gemm_destroy",
-           "adit_attention_static_status", "adit_debug_stamps_selected",
+           "adit_debug_stream_read", "adit_attention_static_status", "adit_debug_stamps_selected",
            "adit_clear_status", "adit_uses_persistent_loop", "adit_debug_wait_limit", "adit_loop_trace_read"]
 
 
@@ -76,6 +76,7 @@ STATIC_SCRATCH_BYTES = 8 << 20
 lib.adit_trace_enable.argtypes = [C.c_void_p, C.c_int]
 lib.adit_trace_read.argtypes = [C.c_void_p, C.POINTER(C.c_int64), C.c_int64]
 lib.adit_trace_read.restype = C.c_int64
+lib.adit_debug_stream_read.argtypes = [C.c_int, C.c_size_t, C.c_int, C.c_int, C.POINTER(C.c_double)]
 lib.adit_attention_static_status.argtypes = [C.c_int]
 lib.adit_debug_stamps_selected.argtypes = [C.c_int] * 4
 lib.adit_clear_status.argtypes = [C.c_void_p]
@@ -247,6 +248,15 @@ def debug_plan(n_tok: int, n_feat: int, k: int, dual: bool = False, sm_count: in
     names = ("tile_tok", "n_ttiles", "n_ftiles", "splits", "stages", "kb_total", "acc_bufs", "issuers", "tmem_cols",
              "smem_bytes", "ring_bytes", "est_ns")
     return dict(zip(names, out))
+
+
+def stream_read_gbs(sm_count: int, n_bytes: int = 1 << 30, iters: int = 5, device: int = 0) -> float:
+    """Read bandwidth (GB/s) of a plain streaming read from `sm_count` SMs."""
+    out = C.c_double(0.0)
+    rc = lib.adit_debug_stream_read(device, n_bytes, sm_count, iters, C.byref(out))
+    if rc != OK:
+        raise AditError(rc)
+    return float(out.value)
 
 
 def upload_prefix_kv(wl: W.Workload, device: int = 0) -> List:

@@ -1476,6 +1476,52 @@ extern "C" int adit_debug_gemm(int device, int n_tok, int n_feat, int k, const v
   return hs ? hs : (p.splits * 1000000 + p.tile_tok * 1000 + p.stages);  // plan, for the test's information
 }
 
+
+// ---------------------------------------------------------------------------------------------
+// Streaming-read microbenchmark: what a plain read of global memory reaches from a given number of SMs
+// (the HBM denominator for runs on a reduced SM budget).
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(512) stream_read_kernel(const uint4* __restrict__ src, size_t n_vec, unsigned* __restrict__ sink) {
+  const size_t per = (n_vec + gridDim.x - 1) / gridDim.x;
+  const size_t lo = (size_t)blockIdx.x * per, hi = lo + per < n_vec ? lo + per : n_vec;
+  unsigned acc = 0;
+  size_t i = lo + threadIdx.x;
+  for (; i + 7 * 512 < hi; i += 8 * 512) {
+    uint4 v[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j)
+      asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v[j].x), "=r"(v[j].y), "=r"(v[j].z), "=r"(v[j].w) : "l"(src + i + (size_t)j * 512));
+#pragma unroll
+    for (int j = 0; j < 8; ++j) acc ^= v[j].x ^ v[j].y ^ v[j].z ^ v[j].w;
+  }
+  for (; i < hi; i += 512) { const uint4 v = src[i]; acc ^= v.x ^ v.y ^ v.z ^ v.w; }
+  if (acc == 0x9e3779b9u) sink[blockIdx.x] = acc;  // (keeps the loads alive; practically never true)
+}
+
+extern "C" int adit_debug_stream_read(int device, size_t bytes, int sm_count, int iters, double* gb_per_s) {
+  if (!gb_per_s || bytes < (1u << 20) || iters < 1 || sm_count < 1) return ADIT_E_INVALID;
+  if (cudaSetDevice(device) != cudaSuccess) return ADIT_E_CUDA;
+  void* buf = nullptr; unsigned* sink = nullptr;
+  if (cudaMalloc(&buf, bytes) != cudaSuccess) return ADIT_E_CUDA;
+  if (cudaMalloc((void**)&sink, 4096 * 4) != cudaSuccess) { cudaFree(buf); return ADIT_E_CUDA; }
+  cudaMemset(buf, 1, bytes);
+  cudaEvent_t a, b;
+  cudaEventCreate(&a); cudaEventCreate(&b);
+  const int grid = sm_count > 4096 ? 4096 : sm_count;
+  stream_read_kernel<<<grid, 512>>>((const uint4*)buf, bytes / 16, sink);
+  cudaEventRecord(a);
+  for (int i = 0; i < iters; ++i) stream_read_kernel<<<grid, 512>>>((const uint4*)buf, bytes / 16, sink);
+  cudaEventRecord(b);
+  cudaError_t e = cudaEventSynchronize(b);
+  float ms = 0.f;
+  if (e == cudaSuccess) e = cudaEventElapsedTime(&ms, a, b);
+  cudaEventDestroy(a); cudaEventDestroy(b);
+  cudaFree(buf); cudaFree(sink);
+  if (e != cudaSuccess || ms <= 0.f) return ADIT_E_CUDA;
+  *gb_per_s = (double)bytes * iters / (ms * 1e-3) / 1e9;
+  return ADIT_OK;
+}
+
 // ---------------------------------------------------------------------------------------------
 // Background GEMM load (stand-in for the VLM stage on the other stream)
 // ---------------------------------------------------------------------------------------------
