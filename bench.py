@@ -623,6 +623,55 @@ def run_colocated(args):
         "results": out}))
 
 
+# ---- lockstep execution with a profiled SM restriction (paper section 4.1.2) ---------------------------
+
+def run_lockstep(args):
+    """VLM stand-in (capped GEMM loop) and the ADiT stage in locksteps on two streams: the offline table of the best
+    SM restriction per (VLM batch, ADiT batch) pair, then a saturated trace with and without the restriction."""
+    import torch
+    from paper_2609_12075_b200 import build, lockstep as LS
+    build.build()
+    from paper_2609_12075_b200 import adit
+    max_batch = args.max_batch
+    cfg = W.PI0
+    pool = 8
+    wl = W.make_workload("lockstep", cfg, seed=7, batch=pool, n_steps=10, prefix_len=[816] * pool, max_prefix_len=816)
+    eng = adit.ADiT(cfg, max_batch=max_batch, max_prefix_len=816)
+    eng.load_weights(W.make_weights(cfg, wl.seed))
+    inputs = {"pi0": {"kv": adit.upload_prefix_kv(wl), "len": wl.prefix_len, "state": torch.from_numpy(wl.state).cuda(),
+                      "noise": torch.from_numpy(wl.noise).cuda(), "steps": wl.n_steps}}
+    stages = LS.GpuStages(adit, {"pi0": eng}, inputs, vlm_iters_per_request=args.vlm_iters)
+    for b in LS.batch_sizes(max_batch):               # record every batch size's launch graph first
+        stages.time_lockstep("pi0", b, b, 0, reps=1)
+    t0 = time.perf_counter()
+    table = LS.SmTable.profile(stages.n_sm, max_batch, lambda vb, ab, cap: stages.time_lockstep("pi0", vb, ab, cap, reps=2))
+    profile_s = time.perf_counter() - t0
+    out = {}
+    for name, tab in (("guarded", table), ("unguarded", LS.SmTable(stages.n_sm))):
+        ex = LS.LockstepExecutor(stages.vlm, stages.adit_stage, max_batch, tab, {"pi0": 156_000})
+        reqs = [LS.Request("pi0", i, 0, payload=i % pool) for i in range(args.requests)]
+        [ex.submit(r) for r in reqs]
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        rec = ex.run()
+        total = time.perf_counter() - t0
+        full = [r.seconds for r in rec if r.vlm_ids and r.adit_ids]
+        out[name] = {"requests": len(reqs), "locksteps": len(rec), "total_s": total, "chunks_per_s": len(reqs) / total,
+                     "mean_lockstep_ms": 1e3 * float(np.mean(full)) if full else None,
+                     "p99_latency_ms": float(np.percentile([r.done_us for r in reqs], 99)) / 1e3}
+    assert eng.poll_status() == 0
+    print(json.dumps({"metric": "lockstep_time_with_profiled_sm_restriction", "unit": "ms", "config": {
+        "expert": "pi0-scale, 816-token prefixes, 10 Euler steps", "max_batch": max_batch,
+        "vlm_stand_in": f"bf16 GEMM 8192x2048x2048 x {args.vlm_iters} per request, grid capped to the restriction",
+        "candidates": "multiples of 8 SMs and no restriction", "n_sm": stages.n_sm, "profile_seconds": profile_s},
+        "table": {f"{vb},{ab}": c for (vb, ab), c in sorted(table.entries.items())},
+        "table_ms": {f"{vb},{ab}": {"best": 1e3 * t[table.entries[(vb, ab)]], "unrestricted": 1e3 * t[0]}
+                     for (vb, ab), t in sorted(table.times.items())},
+        "trace": out, "speedup_guarded_vs_unguarded": out["unguarded"]["total_s"] / out["guarded"]["total_s"]}))
+    stages.close()
+    eng.close()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -632,8 +681,12 @@ def main():
     ap.add_argument("--workload", choices=sorted(WORKLOADS), default=None)
     ap.add_argument("--sm-budget", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--mode", choices=["throughput", "sweep", "colocate"], default="throughput",
-                    help="sweep: latency per sm_budget with/without a concurrent GEMM load; colocate: two experts, two streams")
+    ap.add_argument("--mode", choices=["throughput", "sweep", "colocate", "lockstep"], default="throughput",
+                    help="sweep: latency per sm_budget with/without a concurrent GEMM load; colocate: two experts, two streams; "
+                         "lockstep: VLM stand-in and ADiT in locksteps with the profiled SM restriction")
+    ap.add_argument("--max-batch", type=int, default=4, help="lockstep mode: largest batch admitted per lockstep")
+    ap.add_argument("--vlm-iters", type=int, default=60, help="lockstep mode: GEMM repetitions per request of the VLM stand-in")
+    ap.add_argument("--requests", type=int, default=64, help="lockstep mode: requests in the saturated trace")
     ap.add_argument("--budgets", default="16,32,64,74,148")
     ap.add_argument("--no-trace", action="store_true", help="skip the in-situ timeline of one call")
     ap.add_argument("--no-extra", action="store_true", help="skip the brief runs of the other batch sizes (c3, c4)")
@@ -652,6 +705,8 @@ def main():
         return run_budget_sweep(args)
     if args.mode == "colocate":
         return run_colocated(args)
+    if args.mode == "lockstep":
+        return run_lockstep(args)
     if args.impl == "reference":
         args.steps = 10 if args.steps is None else args.steps
         args.warmup = 1 if args.warmup is None else args.warmup
