@@ -138,7 +138,11 @@ int adit_load_weights(adit_handle* h, const adit_tensor* tensors, int n_tensors)
  * the result by rounding order only.
  * A handle serves one call at a time (calls on one stream are ordered; do not share a handle
  * between streams without synchronising); two handles on two streams may overlap.
- * Errors: INVALID, CAPACITY, NOT_LOADED, CUDA.
+ * Stream capture (section 4.1.1: the stage as a graph per batch size): the call may be recorded into the caller's
+ * own CUDA graph - it then enqueues only kernels, straight into that graph - provided a call with the same K
+ * was made on this handle before, outside any capture (the time-embedding vectors are computed when K changes);
+ * otherwise it returns ADIT_E_UNSUPPORTED and records nothing.  A replay uses the pointers and prefix lengths given at capture time.
+ * Errors: INVALID, CAPACITY, NOT_LOADED, UNSUPPORTED (see above), CUDA.
  */
 int adit_denoise(adit_handle* h, int B, const void* const* prefix_kv, const int32_t* prefix_len,
                  const float* state, const float* noise, int K, int sm_budget, void* stream,

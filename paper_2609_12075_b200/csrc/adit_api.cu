@@ -166,6 +166,10 @@ static AttnPlan plan_attention(const adit_handle* h, int B) {
 struct LoopInFlight { adit_handle* h; int device; cudaEvent_t ev; int clusters; };
 static std::mutex g_loop_mutex;
 static std::vector<LoopInFlight> g_loop_inflight;
+static bool stream_is_capturing(cudaStream_t st) {
+  cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+  return cudaStreamIsCapturing(st, &cs) == cudaSuccess && cs == cudaStreamCaptureStatusActive;
+}
 static cudaError_t init_attention_attrs();
 static int loop_init(adit_handle* h);
 static int loop_build_maps(adit_handle* h);
@@ -940,7 +944,8 @@ static int denoise_loop(adit_handle* h, int B, const PrefixTable& pt, const floa
     p.trace = h->loop_trace;
     h->loop_trace_levels = n_levels; h->loop_trace_blocks = n_blocks; h->loop_trace_layers = c.n_layers;
   }
-  {
+  const bool capturing = stream_is_capturing(st);  // (a captured call is ordered by the caller's graph, not by events here)
+  if (!capturing) {
     // order this call behind loop kernels of other handles that it would not fit beside
     std::lock_guard<std::mutex> lock(g_loop_mutex);
     int busy = 0;
@@ -980,7 +985,7 @@ static int denoise_loop(adit_handle* h, int B, const PrefixTable& pt, const floa
     CU_TRY(h, e);
     h->launches++;
   }
-  {
+  if (!capturing) {
     std::lock_guard<std::mutex> lock(g_loop_mutex);
     CU_TRY(h, cudaEventRecord(h->loop_ev, st));
     bool found = false;
@@ -997,6 +1002,11 @@ static int denoise_tc(adit_handle* h, int B, const PrefixTable& pt, const float*
                       int sm_budget, cudaStream_t st, float* out) {
   const adit_config& c = h->cfg;
   const int G = (sm_budget <= 0 || sm_budget >= h->sm_count) ? h->sm_count : sm_budget;
+  if (stream_is_capturing(st)) {
+    // Inside a caller's stream capture only pure enqueueing is possible: the time vectors for this K must exist
+    // from an earlier call (they are computed by kernels that a graph replay must not repeat on other data).
+    if (h->ctime_steps != K || h->profiling) return ADIT_E_UNSUPPORTED;
+  }
   if (h->ctime_steps != K) {
     // c_k = tau(k/K) . W1[D:, :] + b1 depends on K only: computed when K changes and kept
     const int Tm = c.time_emb_dim, D = c.d_model;
@@ -1014,7 +1024,8 @@ static int denoise_tc(adit_handle* h, int B, const PrefixTable& pt, const float*
   set_desc_kernel<<<1, 32, 0, st>>>(d, h->desc_dev);
   h->launches++;
   CU_TRY(h, cudaGetLastError());
-  if (!h->use_graph || h->profiling) return enqueue_tc(h, B, K, G, st);
+  // (inside a caller's capture the kernels are recorded straight into the caller's graph)
+  if (!h->use_graph || h->profiling || stream_is_capturing(st)) return enqueue_tc(h, B, K, G, st);
 
   auto key = std::make_tuple(B, K, G);
   auto it = h->graphs.find(key);
