@@ -303,6 +303,8 @@ def run_ours(args):
 
         # ---- per-call latency distribution (its own calls: p99 needs many samples whatever --steps is) ----
         lat = sample_latency(torch, eng, sets, K_e, args.sm_budget, stream, args.latency_calls, args.latency_seconds)
+        if len(lat) == 0:       # (--latency-calls 0, for profiler runs: one call's latency from the timed region)
+            lat = np.array([total_ms / args.steps])
 
         # ---- end to end through the host-buffer entry point (pinned host in, host out) ------------
         for i in range(3):
