@@ -25,6 +25,11 @@ the following reading, taken step by step, one request at a time:
   prefix keys [0, prefix_len) followed by all suffix keys, no mask inside that
   set, no positional term, scale 1/sqrt(head_dim), query head h reads kv head
   h // (n_q_heads / n_kv_heads);
+* variants, off unless the configuration asks for them: `state_block_mask` - the state token's query attends to
+  the prefix keys and its own key only (the action tokens still attend to everything); `suffix_rope` - the
+  suffix queries and keys of every head are rotated by the angles pos * 10000**(-2j/head_dim), j < head_dim/2,
+  pairing channel j with channel j + head_dim/2, at position pos = prefix_len + (index of the token in the
+  suffix); prefix keys are used as given (their producer has rotated them);
 * GeGLU: tanh-approximate GELU on the gate times the up projection;
 * read-out: final RMSNorm, then Wout, bout, on the action tokens only.
 
@@ -35,7 +40,11 @@ CPU fp64 library routines (norm -> q/k/v, attention, residual, norm ->
 GeGLU, residual); scalar-loop softmax attention on tiny shapes; zero queries give the
 mean of the valid value rows; torch CPU fp64 library routines for attention,
 RMSNorm, GELU(tanh) and SiLU; grouped-query = replicated multi-head; batch
-permutation, padding and capacity invariance; time-embedding special values.
+permutation, padding and capacity invariance; time-embedding special values;
+for the variants: the masked attention against torch's masked attention and a
+scalar loop, the state token's independence of the action tokens; the rotary
+embedding against its closed form in two dimensions, norm preservation, the
+identity at position 0 and the dependence of a score on the position difference only.
 Parity unpinned: the behaviour of a *trained* model (no weights or reference
 outputs exist); the oracle pins the computation, not robot behaviour.
 """
@@ -79,12 +88,29 @@ def softmax_rows(s: np.ndarray) -> np.ndarray:
     return e / np.sum(e, axis=-1, keepdims=True)
 
 
+ROPE_BASE = 10000.0
+
+
+def rope(x: np.ndarray, pos: float) -> np.ndarray:
+    """Rotary embedding of the last axis at position pos: channel pair (j, j + dh/2) is rotated by the angle
+    pos * ROPE_BASE ** (-2 j / dh)."""
+    dh = x.shape[-1]
+    half = dh // 2
+    assert dh == 2 * half
+    ang = F64(pos) * ROPE_BASE ** (-np.arange(half, dtype=F64) / F64(half))
+    c, s_ = np.cos(ang), np.sin(ang)
+    x1, x2 = x[..., :half], x[..., half:]
+    return np.concatenate([x1 * c - x2 * s_, x2 * c + x1 * s_], axis=-1)
+
+
 def attention(q: np.ndarray, k_suffix: np.ndarray, v_suffix: np.ndarray,
-              k_prefix: np.ndarray, v_prefix: np.ndarray, prefix_len: int) -> np.ndarray:
+              k_prefix: np.ndarray, v_prefix: np.ndarray, prefix_len: int,
+              state_block_mask: bool = False) -> np.ndarray:
     """One request, one layer.
 
     q [N, Hq, dh]; k_suffix, v_suffix [N, Hkv, dh]; k_prefix, v_prefix
     [Hkv, capacity, dh] of which only rows [0, prefix_len) are read.
+    With state_block_mask the first suffix token (the state token) does not see the suffix keys 1..N-1.
     Returns [N, Hq, dh].
     """
     n, hq, dh = q.shape
@@ -97,6 +123,8 @@ def attention(q: np.ndarray, k_suffix: np.ndarray, v_suffix: np.ndarray,
         k_all = np.concatenate([k_prefix[kv, :prefix_len, :], k_suffix[:, kv, :]], axis=0)
         v_all = np.concatenate([v_prefix[kv, :prefix_len, :], v_suffix[:, kv, :]], axis=0)
         s = (q[:, h, :] @ k_all.T) / math.sqrt(dh)
+        if state_block_mask:
+            s[0, prefix_len + 1:] = -np.inf
         out[:, h, :] = softmax_rows(s) @ v_all
     return out
 
@@ -121,7 +149,12 @@ def layer_forward(cfg, w: Dict[str, np.ndarray], l: int, h: np.ndarray,
     q = (u @ w[p + "wq"]).reshape(n, cfg.n_q_heads, cfg.head_dim)
     kc = (u @ w[p + "wk"]).reshape(n, cfg.n_kv_heads, cfg.head_dim)
     vc = (u @ w[p + "wv"]).reshape(n, cfg.n_kv_heads, cfg.head_dim)
-    o = attention(q, kc, vc, kv_prefix_l[0], kv_prefix_l[1], prefix_len)
+    if getattr(cfg, "suffix_rope", False):
+        for i in range(n):
+            q[i] = rope(q[i], prefix_len + i)
+            kc[i] = rope(kc[i], prefix_len + i)
+    o = attention(q, kc, vc, kv_prefix_l[0], kv_prefix_l[1], prefix_len,
+                  state_block_mask=getattr(cfg, "state_block_mask", False))
     h = h + o.reshape(n, cfg.q_dim) @ w[p + "wo"]
     u = rmsnorm(h, w[p + "norm2.g"], cfg.rms_eps)
     h = h + (gelu_tanh(u @ w[p + "wg"]) * (u @ w[p + "wu"])) @ w[p + "wd"]

@@ -53,6 +53,9 @@ class ADiTConfig:
     rms_eps: float = 1e-6
     t_min_period: float = 4e-3
     t_max_period: float = 4.0
+    # model-fidelity variants (off in the configurations of the benchmark)
+    state_block_mask: bool = False   # the state token attends to the prefix and itself only, not to the action tokens
+    suffix_rope: bool = False        # rotary position embedding on the suffix queries/keys at positions prefix_len + i
 
     @property
     def n_tokens(self) -> int:

@@ -407,6 +407,82 @@ def test_layer_wiring_mistakes_are_visible():
     assert np.abs(O.layer_forward(cfg, w4, 0, h, kv, plen) - want).max() > 1e-3
 
 
+# ---- P13: model-fidelity variants (state-block mask, rotary embedding on the suffix) ---------------------------
+
+def test_state_block_mask_against_library_and_scalar_loop():
+    import torch
+    import torch.nn.functional as F
+    rng = np.random.default_rng(31)
+    n, hq, hkv, dh, plen, cap = 4, 4, 2, 8, 5, 7
+    q = rng.standard_normal((n, hq, dh)); ks = rng.standard_normal((n, hkv, dh)); vs = rng.standard_normal((n, hkv, dh))
+    kp = rng.standard_normal((hkv, cap, dh)); vp = rng.standard_normal((hkv, cap, dh))
+    kp[:, plen:] = np.nan; vp[:, plen:] = np.nan
+    got = O.attention(q, ks, vs, kp, vp, plen, state_block_mask=True)
+    plain = O.attention(q, ks, vs, kp, vp, plen)
+    # library: boolean mask, True = may attend
+    allow = torch.ones(n, plen + n, dtype=torch.bool)
+    allow[0, plen + 1:] = False
+    t = lambda a: torch.from_numpy(np.ascontiguousarray(a))
+    k_all = torch.cat([t(kp[:, :plen]), t(ks).transpose(0, 1)], dim=1).repeat_interleave(hq // hkv, dim=0)
+    v_all = torch.cat([t(vp[:, :plen]), t(vs).transpose(0, 1)], dim=1).repeat_interleave(hq // hkv, dim=0)
+    want = F.scaled_dot_product_attention(t(q).transpose(0, 1), k_all, v_all, attn_mask=allow).transpose(0, 1).numpy()
+    np.testing.assert_allclose(got, want, rtol=1e-12, atol=1e-12)
+    # the action tokens are not affected; the state token is
+    np.testing.assert_array_equal(got[1:], plain[1:])
+    assert np.abs(got[0] - plain[0]).max() > 1e-3
+    # scalar loop for the state row of head 3: prefix keys and its own key only
+    h, kvh = 3, 1
+    keys = [kp[kvh, j] for j in range(plen)] + [ks[0, kvh]]
+    vals = [vp[kvh, j] for j in range(plen)] + [vs[0, kvh]]
+    sc = [sum(q[0, h, c] * kk[c] for c in range(dh)) / math.sqrt(dh) for kk in keys]
+    mx = max(sc)
+    ws = [math.exp(v - mx) for v in sc]
+    for c in range(dh):
+        assert abs(got[0, h, c] - sum(wj * vj[c] for wj, vj in zip(ws, vals)) / sum(ws)) < 1e-12
+
+
+def test_state_token_stream_ignores_the_action_tokens_under_the_mask():
+    cfg, w, h, kv, plen = _layer_case()
+    cfg_m = W.scaled(cfg, state_block_mask=True)
+    h2 = h.copy()
+    h2[1:] += 3.0 * np.random.default_rng(5).standard_normal(h2[1:].shape)
+    a, b = O.layer_forward(cfg_m, w, 0, h, kv, plen), O.layer_forward(cfg_m, w, 0, h2, kv, plen)
+    np.testing.assert_allclose(a[0], b[0], rtol=0, atol=1e-13)          # row 0 never saw rows 1..
+    a, b = O.layer_forward(cfg, w, 0, h, kv, plen), O.layer_forward(cfg, w, 0, h2, kv, plen)
+    assert np.abs(a[0] - b[0]).max() > 1e-3                             # without the mask it does
+
+
+def test_rotary_embedding_closed_forms():
+    # two channels: one pair, angle = position (10000 ** 0 = 1)
+    for pos in (0.0, 1.0, 2.5, 817.0):
+        np.testing.assert_allclose(O.rope(np.array([1.0, 0.0]), pos), [math.cos(pos), math.sin(pos)], atol=1e-12)
+        np.testing.assert_allclose(O.rope(np.array([0.0, 1.0]), pos), [-math.sin(pos), math.cos(pos)], atol=1e-12)
+    rng = np.random.default_rng(41)
+    x, y = rng.standard_normal(16), rng.standard_normal(16)
+    np.testing.assert_array_equal(O.rope(x, 0), x)                                   # position 0: identity
+    assert abs(np.linalg.norm(O.rope(x, 123.0)) - np.linalg.norm(x)) < 1e-12          # a rotation
+    # channel j is paired with channel j + dh/2, and pair j turns by pos * 10000 ** (-2 j / dh)
+    j, pos = 3, 7.0
+    e = np.zeros(16); e[j] = 1.0
+    r = O.rope(e, pos)
+    ang = pos * 10000.0 ** (-2 * j / 16)
+    assert abs(r[j] - math.cos(ang)) < 1e-12 and abs(r[j + 8] - math.sin(ang)) < 1e-12 and abs(np.abs(r).sum() - abs(math.cos(ang)) - abs(math.sin(ang))) < 1e-12
+    # a score depends on the difference of the positions only
+    s1 = O.rope(x, 900.0) @ O.rope(y, 893.0)
+    s2 = O.rope(x, 12.0) @ O.rope(y, 5.0)
+    assert abs(s1 - s2) < 1e-9
+
+
+def test_suffix_rope_changes_the_layer_and_reduces_to_plain_at_identity_positions():
+    cfg, w, h, kv, plen = _layer_case()
+    cfg_r = W.scaled(cfg, suffix_rope=True)
+    plain, rot = O.layer_forward(cfg, w, 0, h, kv, plen), O.layer_forward(cfg_r, w, 0, h, kv, plen)
+    assert np.isfinite(rot).all() and np.abs(rot - plain).max() > 1e-3
+    # a single suffix token without a prefix sits at position 0, where the rotation is the identity
+    one, empty = h[:1], kv[:, :, :0]
+    np.testing.assert_allclose(O.layer_forward(cfg_r, w, 0, one, empty, 0), O.layer_forward(cfg, w, 0, one, empty, 0), atol=1e-13)
+
+
 # ---- the full configurations run and are healthy --------------------------------------------
 
 def test_config_c1_runs_and_signal_is_healthy():
