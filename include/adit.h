@@ -18,7 +18,8 @@
  * grouped-query attention (query head h reads kv head h / (n_q_heads / n_kv_heads)), scale
  * 1/sqrt(head_dim), GeGLU MLP with tanh-approximate GELU, final RMSNorm and a linear read-out on
  * the action tokens.  dtype 1 rounds matrix-product operands to bfloat16 and accumulates in fp32;
- * the residual stream and x stay fp32.
+ * the residual stream and x stay fp32.  Two variants of the model can be switched on per handle (section 2.1 leaves
+ * the hand-over and the expert's attention pattern to the model): ADIT_FLAG_STATE_BLOCK_MASK and ADIT_FLAG_SUFFIX_ROPE.
  *
  * All functions return 0 (ADIT_OK) or a negative adit_status.  Nothing is enqueued when an error
  * is returned.  No function throws, aborts or synchronises the host except where stated.
@@ -54,6 +55,9 @@ typedef enum {
 #define ADIT_FLAG_NO_GRAPH 2          /* enqueue kernels one by one instead of replaying a cached launch graph */
 #define ADIT_FLAG_NO_PDL 4            /* no programmatic dependent launch between the loop's kernels */
 #define ADIT_FLAG_MMA_SYNC_ATTENTION 8 /* attention on the legacy mma.sync path instead of tcgen05 (comparison aid) */
+#define ADIT_FLAG_STATE_BLOCK_MASK 32 /* model variant: the state token attends to the prefix and itself only, not to the action tokens */
+#define ADIT_FLAG_SUFFIX_ROPE 64      /* model variant: rotary embedding (pairs j, j + head_dim/2; base 10000) on the suffix queries
+                                         and keys at positions prefix_len[b] + index in the suffix; prefix keys are used as given */
 #define ADIT_FLAG_PERSISTENT_LOOP 16  /* small batches run as one persistent kernel instead of a kernel per phase (see adit_uses_persistent_loop) */
 
 typedef struct adit_handle adit_handle; /* opaque; owns packed weights and a workspace on one device */
@@ -86,7 +90,8 @@ typedef struct {
  * Errors: INVALID (NULL, non-positive sizes, n_q_heads not a multiple of n_kv_heads, odd
  * time_emb_dim), CAPACITY (max_batch > ADIT_MAX_BATCH), UNSUPPORTED (head_dim not in {64,128,256};
  * for dtype bf16 without the reference-kernel flag: a device that is not compute capability 10.x,
- * or d_model/d_ff/head_dim not multiples of 64), CUDA.
+ * or d_model/d_ff/head_dim not multiples of 64; ADIT_FLAG_STATE_BLOCK_MASK together with
+ * ADIT_FLAG_MMA_SYNC_ATTENTION), CUDA.
  */
 int adit_create(const adit_config* cfg, int device, adit_handle** out);
 

@@ -22,6 +22,7 @@ lib = C.CDLL(_LIB_PATH)
 OK, E_INVALID, E_CAPACITY, E_NOT_LOADED, E_UNSUPPORTED, E_CUDA, E_TIMEOUT = 0, -1, -2, -3, -4, -5, -6
 DTYPE_FP32, DTYPE_BF16 = 0, 1
 FLAG_REFERENCE_KERNELS, FLAG_NO_GRAPH, FLAG_NO_PDL, FLAG_MMA_SYNC_ATTENTION, FLAG_PERSISTENT_LOOP = 1, 2, 4, 8, 16
+FLAG_STATE_BLOCK_MASK, FLAG_SUFFIX_ROPE = 32, 64
 MAX_BATCH, MAX_STEPS = 64, 64
 
 EXPORTS = ["adit_create", "adit_load_weights", "adit_denoise", "adit_denoise_host", "adit_destroy",
@@ -97,6 +98,8 @@ class AditError(RuntimeError):
 
 
 def make_config(cfg: W.ADiTConfig, max_batch: int, max_prefix_len: int, flags: int = 0) -> Config:
+    flags |= (FLAG_STATE_BLOCK_MASK if getattr(cfg, "state_block_mask", False) else 0) | \
+             (FLAG_SUFFIX_ROPE if getattr(cfg, "suffix_rope", False) else 0)
     return Config(n_layers=cfg.n_layers, d_model=cfg.d_model, n_q_heads=cfg.n_q_heads, n_kv_heads=cfg.n_kv_heads,
                   head_dim=cfg.head_dim, d_ff=cfg.d_ff, horizon=cfg.horizon, action_dim=cfg.action_dim,
                   state_dim=cfg.state_dim, time_emb_dim=cfg.time_emb_dim, max_batch=max_batch,

@@ -76,6 +76,7 @@ struct adit_handle {
   void *hb = 0, *qkv = 0, *att = 0, *mlp = 0, *ea = 0, *ez = 0;
   int* status_host = 0;  // pinned, device-visible status word
   int* status_dev = 0;   // its device address
+  float2* rope_tab = 0;  // cos/sin per suffix token row and channel pair (variant ADIT_FLAG_SUFFIX_ROPE)
   int64_t launches = 0;
   int last_cuda = 0;
   bool profiling = false;
@@ -190,6 +191,7 @@ static int validate_config(const adit_config* c) {
   if (c->max_batch > ADIT_MAX_BATCH) return ADIT_E_CAPACITY;
   if (c->head_dim != 64 && c->head_dim != 128 && c->head_dim != 256) return ADIT_E_UNSUPPORTED;
   if (c->d_model % 4) return ADIT_E_UNSUPPORTED;
+  if ((c->flags & ADIT_FLAG_STATE_BLOCK_MASK) && (c->flags & ADIT_FLAG_MMA_SYNC_ATTENTION)) return ADIT_E_UNSUPPORTED;
   if (!use_reference_kernels(*c)) {
     if (c->d_model % 64 || c->d_ff % 64) return ADIT_E_UNSUPPORTED;
   }
@@ -244,6 +246,7 @@ extern "C" int adit_create(const adit_config* cfg, int device, adit_handle** out
   ALLOC(h->state_dev, c.max_batch * S * 4); ALLOC(h->noise_dev, Ma * A * 4);
   ALLOC(h->hb, Mx * D * e); ALLOC(h->qkv, Mx * (Q + 2 * KV) * e); ALLOC(h->att, Mx * Q * e);
   ALLOC(h->mlp, Mx * F * e); ALLOC(h->ea, Ma * D * e); ALLOC(h->ez, Ma * D * e);
+  if (c.flags & ADIT_FLAG_SUFFIX_ROPE) ALLOC(h->rope_tab, Mx * (c.head_dim / 2) * 8);
   if (!use_reference_kernels(c)) {
     const int64_t n_ft = (D + tc::TILE_F - 1) / tc::TILE_F;
     ALLOC(h->ssq, n_ft * Mx * 4);
@@ -482,7 +485,8 @@ static void launch_ref_attention(adit_handle* h, cudaStream_t st, const PrefixTa
   const float scale = 1.0f / sqrtf((float)c.head_dim);
 #define LAUNCH_ATT(DH)                                                                                        \
   ref_attention_kernel<T, DH><<<grid, 128, 0, st>>>((const T*)h->qkv, QKV, (T*)h->att, Q, pt, layer, h->n_tok, \
-                                                    c.n_q_heads, c.n_kv_heads, c.max_prefix_len, scale)
+                                                    c.n_q_heads, c.n_kv_heads, c.max_prefix_len, scale,       \
+                                                    (c.flags & ADIT_FLAG_STATE_BLOCK_MASK) ? 1 : 0)
   if (c.head_dim == 64) LAUNCH_ATT(64);
   else if (c.head_dim == 128) LAUNCH_ATT(128);
   else LAUNCH_ATT(256);
@@ -511,6 +515,12 @@ static int denoise_reference(adit_handle* h, int B, const PrefixTable& pt, const
     launch_ref_gemm<float, T, float, EPI_STORE_F32, false>(h, KC_PROLOGUE, st, h->tau, Tm, (const T*)h->W1t, Tm, K, D, Tm,
                                                            EpiArgs{h->ctime, D, nullptr, h->b1, 0});
   }
+  const bool rope = (c.flags & ADIT_FLAG_SUFFIX_ROPE) != 0;
+  if (rope) {
+    ProfScope ps(h, KC_NORM, st);
+    rope_table_kernel<<<(M * (c.head_dim / 2) + 255) / 256, 256, 0, st>>>(h->rope_tab, pt, nullptr, M, h->n_tok, c.head_dim);
+    h->launches++;
+  }
   const float dt = 1.0f / (float)K;
   for (int k = 0; k < K; ++k) {
     {
@@ -533,6 +543,13 @@ static int denoise_reference(adit_handle* h, int B, const PrefixTable& pt, const
       }
       launch_ref_gemm<T, T, T, EPI_STORE, false>(h, KC_GEMM_QKV, st, (const T*)h->hb, D, (const T*)L.wqkv, D, M, QKV, D,
                                                  EpiArgs{h->qkv, QKV, h->rstd, nullptr, 0});
+      if (rope) {
+        ProfScope ps(h, KC_NORM, st);
+        const int nrot = c.n_q_heads + c.n_kv_heads;
+        rope_apply_kernel<T><<<(int)(((int64_t)M * nrot * (c.head_dim / 2) + 127) / 128), 128, 0, st>>>((T*)h->qkv, QKV, h->rope_tab, M, nrot,
+                                                                                                       c.head_dim);
+        h->launches++;
+      }
       launch_ref_attention<T>(h, st, pt, l, B);
       launch_ref_gemm<T, T, float, EPI_RESIDUAL, false>(h, KC_GEMM_O, st, (const T*)h->att, Q, (const T*)L.wo, Q, M, D, Q,
                                                         EpiArgs{h->h, D, nullptr, nullptr, 0});
@@ -679,6 +696,7 @@ static void launch_tc_attention(adit_handle* h, cudaStream_t st, int layer, int 
   a.batch = B; a.n_row_tiles = p.n_row_tiles; a.splits = p.splits;
   a.scale_log2 = 1.4426950408889634f / sqrtf((float)c.head_dim);
   a.part_o = h->att_po; a.part_ml = h->att_pml;
+  a.state_mask = (c.flags & ADIT_FLAG_STATE_BLOCK_MASK) ? 1 : 0;
   const int items = B * c.n_kv_heads * p.n_row_tiles * p.splits;
   const bool capped = Gbudget < h->sm_count;
   const int grid = (capped && items > Gbudget) ? Gbudget : items;
@@ -736,6 +754,13 @@ static int enqueue_tc(adit_handle* h, int B, int K, int G, cudaStream_t st) {
              (const float*)h->Ws, (const float*)h->bs, h->hs, h->hsb, h->rstd_state, B, S, D);
     h->launches++;
   }
+  const bool rope = (c.flags & ADIT_FLAG_SUFFIX_ROPE) != 0;
+  if (rope) {
+    ProfScope ps(h, KC_NORM, st);
+    launch_k(rope_table_kernel, cap((M * (c.head_dim / 2) + 255) / 256), 256, 0, st, pdl, h->rope_tab, PrefixTable{},
+             (const PrefixTable*)&h->desc_dev->pt, M, h->n_tok, c.head_dim);
+    h->launches++;
+  }
   const float dt = 1.0f / (float)K;
   for (int k = 0; k < K; ++k) {
     {
@@ -752,6 +777,13 @@ static int enqueue_tc(adit_handle* h, int B, int K, int G, cudaStream_t st) {
     for (int l = 0; l < c.n_layers; ++l) {
       LayerWeights& L = h->layers[l];
       gemm(KC_GEMM_QKV, L.m_qkv, a_qkv, p_qkv, false, M, QKV, EPI_STORE, h->qkv, QKV, h->rstd, nullptr);
+      if (rope) {
+        ProfScope ps(h, KC_NORM, st);
+        const int nrot = c.n_q_heads + c.n_kv_heads;
+        launch_k(rope_apply_kernel<bf16>, cap(((int64_t)M * nrot * (c.head_dim / 2) + 127) / 128), 128, 0, st, pdl, (bf16*)h->qkv, QKV,
+                 (const float2*)h->rope_tab, M, nrot, c.head_dim);
+        h->launches++;
+      }
       launch_tc_attention(h, st, l, B, G);
       gemm(KC_GEMM_O, L.m_o, a_o, p_o, false, M, D, tc::EPI_RESID_NORM, nullptr, 0, nullptr, nullptr);
       gemm(KC_GEMM_GATEUP, L.m_gu, a_gu, p_gu, true, M, F, EPI_GEGLU, h->mlp, F, h->rstd, nullptr);
@@ -816,7 +848,7 @@ static cudaError_t loop_prepare_dh(int* clusters) {
 static int loop_init(adit_handle* h) {
   const adit_config& c = h->cfg;
   h->loop_ok = false;
-  if (!(c.flags & ADIT_FLAG_PERSISTENT_LOOP)) return ADIT_OK;
+  if (!(c.flags & ADIT_FLAG_PERSISTENT_LOOP) || (c.flags & ADIT_FLAG_SUFFIX_ROPE)) return ADIT_OK;
   const int D = c.d_model, F = c.d_ff, Q = c.n_q_heads * c.head_dim, KV = c.n_kv_heads * c.head_dim, QKV = Q + 2 * KV;
   const int G = c.n_q_heads / c.n_kv_heads;
   if (D % 128 || F % 128 || QKV % 128 || Q % 128 || (128 % G) || !h->q_tma) return ADIT_OK;
@@ -930,6 +962,7 @@ static int denoise_loop(adit_handle* h, int B, const PrefixTable& pt, const floa
   p.Wout = h->Wout; p.bout = h->bout; p.b2 = h->b2; p.hsb = h->hsb;
   p.counters = h->loop_counters; p.status = h->status_dev; p.xscratch = h->loop_scratch;
   p.timeout_ns = h->wait_limit_ns; p.debug_skip_level = h->debug_skip_level;
+  p.state_mask = (c.flags & ADIT_FLAG_STATE_BLOCK_MASK) ? 1 : 0;
   const int n_levels = K * (3 + 5 * c.n_layers), n_blocks = clusters * loop::CS;
   p.trace = nullptr;
   if (h->tracing) {

@@ -335,6 +335,14 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
           for (int j = 0; j < 64; ++j)
             if (key0 + j >= total) sc[j] = -INFINITY;
         }
+        // variant: the state token's rows (token 0 of the request: rows 0 .. G-1 of row tile 0) see the prefix and
+        // the state token's own key only
+        const bool state_row = a.state_mask && rt * TC_ROWS + row < G;
+        if (state_row && key0 + KEY_BLOCK > plen + 1) {
+#pragma unroll
+          for (int j = 0; j < 64; ++j)
+            if (key0 + j > plen) sc[j] = -INFINITY;
+        }
         // (four independent chains: a single thread per scheduler cannot hide the latency of one long chain)
         float mx[4] = {sc[0], sc[1], sc[2], sc[3]};
 #pragma unroll
@@ -375,6 +383,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
           if (!warp_wait(&pv_done[q & 1], (q >> 1) & 1)) { ok = false; break; }
         }
         uint8_t* sPn = sP + s * P_BYTES;
+        // (a key range whose keys are all masked for this row leaves the reference maximum at -inf: subtract 0 then,
+        // so that the probabilities are exp2(-inf) = 0 and not NaN)
+        const float m_sub = m_ref == -INFINITY ? 0.f : m_ref;
         // probabilities -> bf16 -> shared memory (row = 128 bytes = 8 swizzled chunks)
         float rs[4] = {0.f, 0.f, 0.f, 0.f};  // partial row sums, added up in a fixed order
 #pragma unroll
@@ -382,7 +393,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
           uint32_t w[4];
 #pragma unroll
           for (int q = 0; q < 4; ++q) {
-            const float p0 = ex2(fmaf(sc[c * 8 + 2 * q], a.scale_log2, -m_ref)), p1 = ex2(fmaf(sc[c * 8 + 2 * q + 1], a.scale_log2, -m_ref));
+            const float p0 = ex2(fmaf(sc[c * 8 + 2 * q], a.scale_log2, -m_sub)), p1 = ex2(fmaf(sc[c * 8 + 2 * q + 1], a.scale_log2, -m_sub));
             rs[q] += p0 + p1;
             w[q] = pack_bf16(p0, p1);
           }

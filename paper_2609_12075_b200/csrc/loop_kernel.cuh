@@ -100,6 +100,7 @@ struct LoopParams {
   uint32_t* counters;  // [LV_COUNT] level counters, [LV_COUNT] abort word; zeroed before every call
   int* status;         // host-visible status word
   unsigned long long timeout_ns;
+  int state_mask;        // variant: the state token attends to the prefix and itself only
   int debug_skip_level;  // test aid: the level type whose first flag increment of block 0 is withheld (-1: none)
   unsigned long long* trace;  // optional [level][block][8] timestamps
 };
@@ -817,6 +818,13 @@ __device__ void role_epilogue(const Ctx& c) {
             for (int j = 0; j < 64; ++j)
               if (j >= nvalid) sc[j] = -INFINITY;
           }
+          // variant: the state token's rows (rows 0 .. G-1 of row tile 0) see, of the suffix, only the state token's key
+          if (p.state_mask && a.rt * 128 + row < G && blk >= a.npb) {
+            const int first = (blk - a.npb) * attn::KEY_BLOCK;
+#pragma unroll
+            for (int j = 0; j < 64; ++j)
+              if (first + j > 0) sc[j] = -INFINITY;
+          }
           float mx[4] = {sc[0], sc[1], sc[2], sc[3]};
 #pragma unroll
           for (int j = 4; j < 64; j += 4) {
@@ -852,13 +860,14 @@ __device__ void role_epilogue(const Ctx& c) {
             if (!warp_wait(c, &ms->pv_done[q & 1], (q >> 1) & 1u)) { ok = false; break; }
           }
           uint8_t* sPn = c.pool + OFF_P + s * P_BYTES;
+          const float m_sub = m_ref == -INFINITY ? 0.f : m_ref;  // (all keys of the range masked for this row: exp2(-inf) = 0)
           float rs4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
           for (int ch = 0; ch < 8; ++ch) {
             uint32_t w[4];
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
-              const float p0 = ex2f(fmaf(sc[ch * 8 + 2 * q], p.scale_log2, -m_ref)), p1 = ex2f(fmaf(sc[ch * 8 + 2 * q + 1], p.scale_log2, -m_ref));
+              const float p0 = ex2f(fmaf(sc[ch * 8 + 2 * q], p.scale_log2, -m_sub)), p1 = ex2f(fmaf(sc[ch * 8 + 2 * q + 1], p.scale_log2, -m_sub));
               rs4[q] += p0 + p1;
               w[q] = attn::pack_bf16(p0, p1);
             }

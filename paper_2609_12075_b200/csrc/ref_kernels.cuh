@@ -123,7 +123,8 @@ __global__ void __launch_bounds__(256) rowstats_kernel(const float* __restrict__
 template <typename T, int DH>
 __global__ void __launch_bounds__(128) ref_attention_kernel(const T* __restrict__ qkv, int ldqkv, T* __restrict__ att,
                                                             int ldatt, PrefixTable pt, int layer, int n_tokens,
-                                                            int n_q_heads, int n_kv_heads, int p_cap, float scale) {
+                                                            int n_q_heads, int n_kv_heads, int p_cap, float scale,
+                                                            int state_mask) {
   constexpr int E = DH / 32;
   const int tok = blockIdx.x, hq = blockIdx.y, b = blockIdx.z;
   const int kvh = hq / (n_q_heads / n_kv_heads);
@@ -144,6 +145,7 @@ __global__ void __launch_bounds__(128) ref_attention_kernel(const T* __restrict_
   }
   float mx = -INFINITY, l = 0.f;
   for (int key = warp; key < total; key += 4) {
+    if (state_mask && tok == 0 && key > plen) break;  // the state token sees the prefix and itself only
     const T *kr, *vr;
     if (key < plen) {
       kr = pk + (int64_t)key * DH;
@@ -292,6 +294,47 @@ __global__ void __launch_bounds__(256) final_kernel(const float* __restrict__ h,
         if (out) out[(int64_t)m * A + j] = xn;
       }
     }
+  }
+}
+
+
+// ---------------------------------------------------------------------------------------------
+// Rotary embedding on the suffix queries and keys (variant ADIT_FLAG_SUFFIX_ROPE).
+// Once per call: cos/sin of pos * 10000^(-2j/dh) for every suffix token row, pos = prefix_len[b] + index in the
+// suffix, computed in fp64 and kept as fp32 pairs [row][dh/2].  After every Q/K/V projection: channel pairs
+// (j, j + dh/2) of every query head and key head of the row are rotated in place.
+// ---------------------------------------------------------------------------------------------
+__global__ void rope_table_kernel(float2* __restrict__ tab, PrefixTable pt, const PrefixTable* __restrict__ ptp, int n_rows,
+                                  int n_tokens, int dh) {
+  ptx::pdl_launch_dependents();
+  ptx::pdl_wait_prior_grids();
+  const int half = dh / 2;
+  const PrefixTable& t = ptp ? *ptp : pt;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < (int64_t)n_rows * half; i += (int64_t)gridDim.x * blockDim.x) {
+    const int row = (int)(i / half), j = (int)(i % half);
+    const int b = row / n_tokens;
+    const double pos = (double)(t.len[b] + (row - b * n_tokens));
+    const double ang = pos * pow(10000.0, -(double)j / (double)half);
+    tab[i] = make_float2((float)cos(ang), (float)sin(ang));
+  }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(128) rope_apply_kernel(T* __restrict__ qkv, int ldqkv, const float2* __restrict__ tab, int n_rows,
+                                                         int n_rot_heads, int dh) {
+  ptx::pdl_launch_dependents();
+  ptx::pdl_wait_prior_grids();
+  const int half = dh / 2;
+  const int64_t n = (int64_t)n_rows * n_rot_heads * half;   // query heads then key heads are contiguous in a row
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
+    const int j = (int)(i % half);
+    const int hd = (int)((i / half) % n_rot_heads);
+    const int row = (int)(i / ((int64_t)half * n_rot_heads));
+    T* p = qkv + (int64_t)row * ldqkv + hd * dh;
+    const float2 cs = tab[(int64_t)row * half + j];
+    const float x1 = to_f32(p[j]), x2 = to_f32(p[j + half]);
+    p[j] = from_f32<T>(x1 * cs.x - x2 * cs.y);
+    p[j + half] = from_f32<T>(x2 * cs.x + x1 * cs.y);
   }
 }
 
