@@ -60,6 +60,9 @@ struct adit_handle {
   bf16* hsb = 0;                    // bf16 copy of the state token rows
   int ctime_steps = 0; // the K for which ctime currently holds the time vectors (tensor-core path)
   CallDesc* desc_dev = 0;          // per-call descriptor read by the kernels of the launch graph
+  KvMaps* kvmaps_dev = 0;          // per-call tensor maps of the prefix caches (tensor-core attention)
+  CUtensorMap m_sfx;               // this step's K/V rows in the qkv workspace: boxes of 64 rows x 64 channels; its row
+  int64_t m_sfx_rows = 0;          //   extent is the call's token count, so rows left by an earlier, larger call read as zeros
   cudaStream_t cap_stream = 0;     // stream used only to capture launch graphs
   bool use_graph = true, use_pdl = true;
   // optional timeline: per launch, every block's start/end timestamp
@@ -164,6 +167,16 @@ static AttnPlan plan_attention(const adit_handle* h, int B) {
   return p;
 }
 
+// Writes the call's prefix-cache tensor maps to device memory (they arrive as a by-value parameter, so the caller's
+// host arrays are consumed at enqueue time) and releases them to the copy engine's proxy.
+__global__ void set_kvmaps_kernel(const __grid_constant__ KvMaps m, KvMaps* __restrict__ dst, int n) {
+  const uint4* src = reinterpret_cast<const uint4*>(&m);
+  uint4* d = reinterpret_cast<uint4*>(dst);
+  for (int i = threadIdx.x; i < n * (int)(sizeof(CUtensorMap) / 16); i += blockDim.x) d[i] = src[i];
+  __syncthreads();
+  if (threadIdx.x == 0) ptx::tensormap_release();
+}
+
 struct LoopInFlight { adit_handle* h; int device; cudaEvent_t ev; int clusters; };
 static std::mutex g_loop_mutex;
 static std::vector<LoopInFlight> g_loop_inflight;
@@ -173,6 +186,7 @@ static bool stream_is_capturing(cudaStream_t st) {
 }
 static cudaError_t init_attention_attrs();
 static int loop_init(adit_handle* h);
+static bool make_map_prefix(CUtensorMap* m, const void* base, int dh, int plen, int p_cap, int64_t planes);
 static int loop_build_maps(adit_handle* h);
 static const int ROW_PAD = 320;  // rows beyond the last token that a token tile (<= 256 wide, remapped rows) may touch
 static bool use_reference_kernels(const adit_config& c) {
@@ -265,6 +279,9 @@ extern "C" int adit_create(const adit_config* cfg, int device, adit_handle** out
     ALLOC(h->att_po, worst * c.head_dim * 4);
     ALLOC(h->att_pml, worst * 2 * 4);
     ALLOC(h->desc_dev, sizeof(CallDesc));
+    ALLOC(h->kvmaps_dev, sizeof(KvMaps));
+    if (!tc::make_map_bf16(&h->m_sfx, h->qkv, (uint64_t)Mx, (uint64_t)(Q + 2 * KV), attn::KEY_BLOCK)) return fail(ADIT_E_CUDA);
+    h->m_sfx_rows = Mx;
     h->q_tma = tc::make_map_q(&h->m_q, h->qkv, (uint64_t)Mx, (uint64_t)(Q + 2 * KV), (uint32_t)c.head_dim,
                               (uint32_t)c.n_q_heads, (uint32_t)(c.n_q_heads / c.n_kv_heads));
     if (!h->q_tma) memset(&h->m_q, 0, sizeof(h->m_q));
@@ -655,10 +672,16 @@ static void launch_attn_dh(adit_handle* h, const attn::AttnArgs& a_in, const Att
   attn::AttnArgs a = a_in;
   a.trace = trace_slot(h, KC_ATTENTION, grid);
   a.status = h->status_dev;
+  a.kv_maps = h->kvmaps_dev->pk;
   a.q_tma = h->q_tma ? 1 : 0;
+  // The last suffix block of the call reaches past its last token: the map ends there, so the copy engine fills those
+  // key rows with zeros (their probabilities are zero, but 0 x a stale non-finite value would not be).
+  const int64_t rows = (int64_t)a.batch * a.n_tokens;
+  if (rows != h->m_sfx_rows && tc::make_map_bf16(&h->m_sfx, h->qkv, (uint64_t)rows, (uint64_t)a.ldqkv, attn::KEY_BLOCK))
+    h->m_sfx_rows = rows;
   if (!(h->cfg.flags & ADIT_FLAG_MMA_SYNC_ATTENTION))
     launch_k(pick_attn_kernel<DH>(a.trace != nullptr, a.splits > 1, a.q_tma != 0), grid, attn::TC_THREADS,
-             attn::attn_tc_smem_bytes<DH>(), st, pdl, h->m_q, a, (const PrefixTable*)&h->desc_dev->pt);
+             attn::attn_tc_smem_bytes<DH>(), st, pdl, h->m_q, h->m_sfx, a, (const PrefixTable*)&h->desc_dev->pt);
   else if (p.nw == 2)
     launch_k(attn::attn_mma_kernel<DH, 2>, grid, 64, attn::attn_smem_bytes<DH, 2>(), st, pdl, a,
              (const PrefixTable*)&h->desc_dev->pt);
@@ -945,6 +968,9 @@ static int denoise_loop(adit_handle* h, int B, const PrefixTable& pt, const floa
     }
   }
   p.maps = h->maps_dev;
+  // (rows past the call's last token read as zeros: a masked key's V row must be finite for P V)
+  if (!tc::make_map_bf16(&p.kv2d, h->qkv, (uint64_t)B * h->n_tok, (uint64_t)(c.n_q_heads + 2 * c.n_kv_heads) * c.head_dim, attn::KEY_BLOCK))
+    return ADIT_E_CUDA;
   for (int i = 0; i < loop::G_COUNT; ++i) p.g[i] = h->loop_g[i];
   p.L = c.n_layers; p.K = K; p.D = D; p.F = c.d_ff; p.n_q_heads = c.n_q_heads; p.n_kv_heads = c.n_kv_heads;
   p.n_tok = h->n_tok; p.horizon = Ta; p.A = A; p.B = B; p.M = B * h->n_tok; p.Ma = B * Ta;
@@ -1056,6 +1082,16 @@ static int denoise_tc(adit_handle* h, int B, const PrefixTable& pt, const float*
   d.pt = pt; d.state = state; d.noise = noise; d.out = out;
   set_desc_kernel<<<1, 32, 0, st>>>(d, h->desc_dev);
   h->launches++;
+  if (!(c.flags & ADIT_FLAG_MMA_SYNC_ATTENTION)) {
+    KvMaps km;
+    const int64_t planes = (int64_t)c.n_layers * 2 * c.n_kv_heads;
+    for (int b = 0; b < B; ++b) {
+      if (pt.len[b] > 0) { if (!make_map_prefix(&km.pk[b], pt.kv[b], c.head_dim, pt.len[b], c.max_prefix_len, planes)) return ADIT_E_CUDA; }
+      else km.pk[b] = h->m_sfx;  // never used (no prefix block): any valid map
+    }
+    set_kvmaps_kernel<<<1, 128, 0, st>>>(km, h->kvmaps_dev, B);
+    h->launches++;
+  }
   CU_TRY(h, cudaGetLastError());
   // (inside a caller's capture the kernels are recorded straight into the caller's graph)
   if (!h->use_graph || h->profiling || stream_is_capturing(st)) return enqueue_tc(h, B, K, G, st);
@@ -1343,13 +1379,14 @@ template <int DH>
 static cudaError_t attention_launch_dh(const attn::AttnArgs& a, int nw, int grid, int merge_grid, int64_t n_qrows,
                                        const PrefixTable* pt_dev, cudaStream_t st) {
   (void)nw;
-  CUtensorMap mq;
+  CUtensorMap mq, msfx;
+  if (!tc::make_map_bf16(&msfx, a.qkv, (uint64_t)a.batch * a.n_tokens, (uint64_t)a.ldqkv, attn::KEY_BLOCK)) return cudaErrorInvalidValue;
   attn::AttnArgs b = a;
   b.q_tma = tc::make_map_q(&mq, a.qkv, (uint64_t)a.batch * a.n_tokens, (uint64_t)a.ldqkv, DH, (uint32_t)a.n_q_heads,
                            (uint32_t)(a.n_q_heads / a.n_kv_heads)) ? 1 : 0;
   if (!b.q_tma) memset(&mq, 0, sizeof(mq));
   auto kern = pick_attn_kernel<DH>(b.dbg != nullptr, b.splits > 1, b.q_tma != 0);
-  kern<<<grid, attn::TC_THREADS, attn::attn_tc_smem_bytes<DH>(), st>>>(mq, b, pt_dev);
+  kern<<<grid, attn::TC_THREADS, attn::attn_tc_smem_bytes<DH>(), st>>>(mq, msfx, b, pt_dev);
   if (a.splits > 1)
     (a.splits > 4 ? attn::attn_merge_kernel<DH, bf16, 16, (DH >= 128 ? 2 : 1)> : attn::attn_merge_kernel<DH, bf16, 4>)
         <<<a.splits > 4 ? merge_grid * (DH >= 128 ? 2 : 1) : merge_grid, 128, 0, st>>>(
@@ -1360,7 +1397,8 @@ static cudaError_t attention_launch_dh(const attn::AttnArgs& a, int nw, int grid
 // Enqueue attention on `st`.  `scratch` holds the key-split partials (attention_scratch_bytes) and
 // `pt_dev` the device copy of the prefix table (written here by a small kernel).
 static cudaError_t attention_enqueue(const AttnProblem& q, const PrefixTable& pt, const void* qkv, void* out_att,
-                                     unsigned char* scratch, PrefixTable* pt_dev, int* status_dev, cudaStream_t st) {
+                                     unsigned char* scratch, PrefixTable* pt_dev, int* status_dev, KvMaps* maps_dev,
+                                     cudaStream_t st) {
   const int G = q.n_q_heads / q.n_kv_heads, R = q.n_tokens * G;
   const int nw = R <= 32 ? 2 : 4;
   const int Q = q.n_q_heads * q.head_dim;
@@ -1375,6 +1413,19 @@ static cudaError_t attention_enqueue(const AttnProblem& q, const PrefixTable& pt
   a.part_ml = (float*)(scratch + rows * q.head_dim * 4);  // (the bf16 partials use half of the first region)
   a.status = status_dev;  // cleared by the table kernel, set to ADIT_E_TIMEOUT by a wait that runs out
   set_table_kernel<<<1, 32, 0, st>>>(pt, pt_dev, status_dev);
+  {
+    KvMaps km;
+    const int64_t planes = (int64_t)(q.layer + 1) * 2 * q.n_kv_heads;   // the cache is indexed up to `layer`
+    CUtensorMap any;
+    if (!tc::make_map_bf16(&any, qkv, (uint64_t)q.B * q.n_tokens, (uint64_t)(Q + 2 * q.n_kv_heads * q.head_dim), attn::KEY_BLOCK))
+      return cudaErrorInvalidValue;
+    for (int b = 0; b < q.B; ++b) {
+      if (pt.len[b] > 0) { if (!make_map_prefix(&km.pk[b], pt.kv[b], q.head_dim, pt.len[b], q.p_cap, planes)) return cudaErrorInvalidValue; }
+      else km.pk[b] = any;
+    }
+    set_kvmaps_kernel<<<1, 128, 0, st>>>(km, maps_dev, q.B);
+    a.kv_maps = maps_dev->pk;
+  }
   const int grid = q.B * q.n_kv_heads * a.n_row_tiles * q.splits;
   const int64_t n_qrows = (int64_t)q.B * q.n_tokens * q.n_q_heads;
   const int mg = (int)((n_qrows + 3) / 4);
@@ -1395,11 +1446,12 @@ extern "C" int adit_debug_attention(int device, int B, int n_tokens, int n_q_hea
   unsigned char* scratch = nullptr;
   PrefixTable* pt_dev = nullptr;
   const size_t nb = attention_scratch_bytes(q);
-  if (cudaMalloc((void**)&pt_dev, sizeof(PrefixTable) + 16) != cudaSuccess) return ADIT_E_CUDA;
+  const size_t maps_off = (sizeof(PrefixTable) + 16 + 255) / 256 * 256;
+  if (cudaMalloc((void**)&pt_dev, maps_off + sizeof(KvMaps)) != cudaSuccess) return ADIT_E_CUDA;
   if (nb && cudaMalloc((void**)&scratch, nb) != cudaSuccess) { cudaFree(pt_dev); return ADIT_E_CUDA; }
   cudaStream_t st = (cudaStream_t)stream;
   int* status_dev = (int*)((unsigned char*)pt_dev + sizeof(PrefixTable));
-  cudaError_t e = attention_enqueue(q, pt, qkv, out_att, scratch, pt_dev, status_dev, st);
+  cudaError_t e = attention_enqueue(q, pt, qkv, out_att, scratch, pt_dev, status_dev, (KvMaps*)((unsigned char*)pt_dev + maps_off), st);
   if (e == cudaSuccess) e = cudaStreamSynchronize(st);
   int hs = 0;
   if (e == cudaSuccess) e = cudaMemcpy(&hs, status_dev, 4, cudaMemcpyDeviceToHost);
@@ -1414,7 +1466,9 @@ extern "C" int adit_debug_attention(int device, int B, int n_tokens, int n_q_hea
 // Scratch (key-split partials + the device copy of the prefix table) lives in a fixed array that every
 // GPU loading this library holds until the process exits.
 // ---------------------------------------------------------------------------------------------
-static __device__ __align__(256) unsigned char g_static_scratch[ADIT_STATIC_SCRATCH_BYTES + sizeof(PrefixTable) + 256];
+// [key-split partials | prefix table, status word (within 1 KB) | the call's prefix-cache tensor maps]
+static __device__ __align__(256) unsigned char g_static_scratch[ADIT_STATIC_SCRATCH_BYTES + 1024 + sizeof(KvMaps)];
+static_assert(sizeof(PrefixTable) + 16 <= 1024, "table and status word must fit their slot");
 static unsigned char* g_static_scratch_addr[64] = {};  // device address of the array, per device ordinal
 
 extern "C" int adit_attention_static(int device, int B, int n_tokens, int n_q_heads, int n_kv_heads, int head_dim,
@@ -1440,7 +1494,8 @@ extern "C" int adit_attention_static(int device, int B, int n_tokens, int n_q_he
   // Nothing in the scratch has to start at zero: every (split, row) partial that the merge reads is
   // written by the attention kernel of the same call, empty splits included.
   int* status_dev = (int*)(base + ADIT_STATIC_SCRATCH_BYTES + sizeof(PrefixTable));  // inside the array's last 256 bytes
-  cudaError_t e = attention_enqueue(q, pt, qkv, out_att, base, pt_dev, status_dev, (cudaStream_t)stream);
+  cudaError_t e = attention_enqueue(q, pt, qkv, out_att, base, pt_dev, status_dev, (KvMaps*)(base + ADIT_STATIC_SCRATCH_BYTES + 1024),
+                                    (cudaStream_t)stream);
   return e == cudaSuccess ? ADIT_OK : ADIT_E_CUDA;
 }
 

@@ -34,6 +34,7 @@ struct AttnArgs {
   int q_tma;        // tcgen05 kernel: the query tile comes in by TMA (group size divides 128)
   unsigned long long* dbg;  // optional [grid][16] phase stamps of the tcgen05 kernel (test aid)
   int* status;      // device-visible status word (ADIT_E_TIMEOUT = -6 on an expired wait); may be null
+  const CUtensorMap* kv_maps;  // tcgen05 kernel: per-request tensor maps of the prefix caches (device memory, see KvMaps)
   int state_mask;   // variant: the first suffix token of a request attends to the prefix and itself only
 };
 

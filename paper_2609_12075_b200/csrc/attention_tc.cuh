@@ -12,9 +12,11 @@
 // O is only rescaled when a row's running maximum grows by more than 2^8 (the reference maximum is kept
 // otherwise), which keeps the TMEM read-modify-write off the common path.
 //
-// K and V blocks are brought in by two loader warps each with 16-byte cp.async copies straight into the
-// 128-byte-swizzled layout the MMA descriptors expect; rows outside the valid key list are written
-// as zeros and their scores masked to -inf, so padding rows of the caller's cache are never read.
+// The key list of a request is [prefix 0..P_b), padded with masked keys to a multiple of 64, then the suffix keys:
+// every 64-key block is then either a box of the request's prefix cache or a box of this step's suffix K/V rows, and
+// both come in by TMA (cp.async.bulk.tensor, 128-byte swizzle = the layout the MMA descriptors expect), issued by
+// one thread per operand.  The prefix cache is described by a per-request tensor map whose row extent is the prefix
+// length: rows at or beyond it are never read (the copy engine writes zeros), and their scores are masked to -inf.
 // The K and V rings (two stages each) are released separately - a K stage as soon as its Q K^T has
 // completed, a V stage after its P V - and P is double-buffered, so the softmax of block n only
 // depends on the tensor core through S(n) and, when a row maximum forces a rescale of O, P V(n - 1).
@@ -29,7 +31,7 @@ namespace adit {
 namespace attn {
 
 constexpr int TC_ROWS = 128;
-constexpr int TC_LOADERS = 64;   // loader threads per operand (warps 4-5: K, warps 6-7: V)
+constexpr int TC_LOADERS = 64;   // threads per operand that help to stage a key split's output (warps 4-5, 6-7); thread 0 of each group issues the operand's copies
 constexpr int TC_THREADS = 320;  // warps 0-3 softmax, 4-7 loaders, 8 issuer of Q K^T (+ TMEM owner), 9 issuer of P V
 
 template <int DH>
@@ -51,7 +53,8 @@ __device__ __forceinline__ uint32_t swz(int r, int c) { return (uint32_t)(r * 12
 // PARTIAL: the key list of a row tile is split over several blocks (a.splits > 1): unnormalised partial outputs.
 // QTMA: the query tile comes in by TMA (the usual case); otherwise by per-thread copies.
 template <int DH, bool INSTR = false, bool PARTIAL = false, bool QTMA = true>
-__global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, AttnArgs a,
+__global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_constant__ CUtensorMap map_q,
+                                                                const __grid_constant__ CUtensorMap map_sfx, AttnArgs a,
                                                                 const PrefixTable* __restrict__ ptp) {
   constexpr int KV_BYTES = KEY_BLOCK * DH * 2;
   constexpr int Q_BYTES = TC_ROWS * DH * 2;
@@ -84,8 +87,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
 
   if (tid == 0) {
     for (int s = 0; s < 2; ++s) {
-      ptx::mbar_init(&k_full[s], TC_LOADERS);
-      ptx::mbar_init(&v_full[s], TC_LOADERS);
+      ptx::mbar_init(&k_full[s], 1);  // the loading thread's expect-tx arrival; the copies count the bytes
+      ptx::mbar_init(&v_full[s], 1);
       ptx::mbar_init(&k_empty[s], 1);
       ptx::mbar_init(&v_empty[s], 1);
       ptx::mbar_init(&s_full[s], 1);
@@ -128,8 +131,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
     const int kvh = t % a.n_kv_heads;
     const int b = t / a.n_kv_heads;
     const int plen = pt.len[b];
-    const int total = plen + a.n_tokens;
-    const int nkb = (total + KEY_BLOCK - 1) / KEY_BLOCK;
+    const int npb = (plen + KEY_BLOCK - 1) / KEY_BLOCK;                       // prefix blocks (the last one padded)
+    const int nkb = npb + (a.n_tokens + KEY_BLOCK - 1) / KEY_BLOCK;           // + suffix blocks
     const int kb0 = PARTIAL ? (int)((int64_t)split * nkb / n_splits) : 0;
     const int kb1 = PARTIAL ? (int)((int64_t)(split + 1) * nkb / n_splits) : nkb;
     const int nb = kb1 - kb0;
@@ -174,53 +177,38 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
     if (warp >= 4 && warp < 8) {
       // ------------------------------ K loaders (warps 4-5) and V loaders (warps 6-7) ------------------------------
       const int which = warp >= 6 ? 1 : 0;
-      const bf16* pref = (const bf16*)pt.kv[b] + ((int64_t)(a.layer * 2 + which) * a.n_kv_heads + kvh) * a.p_cap * DH;
-      const int lt = tid - (which ? 192 : 128);  // 0..63
       uint64_t* empty_bar = which ? v_empty : k_empty;
       uint64_t* full_bar = which ? v_full : k_full;
       uint8_t* ring = which ? sV : sK;
-      for (int i = 0; i < nb && ok; ++i) {
-        const uint32_t n = kv_cnt + i;
-        const int s = n & 1;
-        if (lane == 0 && !ptx::mbar_wait(&empty_bar[s], ((n >> 1) & 1) ^ 1)) ok = false;
-        ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
-        if (!ok) break;
-        for (int spin = 0; spin < 4096 && !ptx::mbar_try_wait(&empty_bar[s], ((n >> 1) & 1) ^ 1); ++spin) {}
-        uint8_t* dst = ring + s * KV_BYTES;
-        // thread lt copies 16-byte piece c of rows r0, r0 + RPP, ...
-        constexpr int CPR = DH / 8, RPP = TC_LOADERS / CPR;
-        const int c = lt % CPR, r0 = lt / CPR;
-        const int key0 = (kb0 + i) * KEY_BLOCK;
-        const uint32_t box = (uint32_t)(c >> 3) * (KEY_BLOCK * 128);
-        if (key0 + KEY_BLOCK <= plen) {  // the whole block lies in the prefix cache: no per-row decisions
-          const bf16* src = pref + (int64_t)(key0 + r0) * DH + c * 8;
+      if (tid == (which ? 192 : 128)) {
+        // one thread per operand issues the copies: dh / 64 boxes of 64 keys x 64 channels per block
+        const int plane = (a.layer * 2 + which) * a.n_kv_heads + kvh;
+        const CUtensorMap* pm = a.kv_maps + b;
+        if (npb > 0 && kb0 < npb) ptx::tensormap_acquire(pm);
+        for (int i = 0; i < nb && ok; ++i) {
+          const uint32_t n = kv_cnt + i;
+          const int s = n & 1;
+          if (!ptx::mbar_wait(&empty_bar[s], ((n >> 1) & 1) ^ 1)) { ok = false; break; }
+          uint8_t* dst = ring + s * KV_BYTES;
+          const int blk = kb0 + i;
+          ptx::mbar_arrive_expect_tx(&full_bar[s], KV_BYTES);
+          if (blk < npb) {
 #pragma unroll
-          for (int p = 0; p < KEY_BLOCK / RPP; ++p)
-            cp_async16(dst + box + swz(r0 + p * RPP, c & 7), src + (int64_t)p * RPP * DH);
-        } else {
-          // Rows [0, np) of the block come from the prefix cache, [np, nt) from this step's suffix, the rest is
-          // zero.  This thread's rows are r0, r0 + RPP, ...: three short loops with running pointers (this code runs
-          // once or twice per work item on a warp with nothing to overlap it: every instruction counts).
-          const int np = min(max(plen - key0, 0), KEY_BLOCK), nt = min(total - key0, KEY_BLOCK);
-          int r = r0;
-          const bf16* src = pref + (int64_t)(key0 + r0) * DH + c * 8;
-#pragma unroll 4
-          for (; r < np; r += RPP, src += RPP * DH) cp_async16(dst + box + swz(r, c & 7), src);
-          if (!waited) { ptx::pdl_wait_prior_grids(); waited = true; }  // only the suffix rows depend on the preceding grid
-          src = a.qkv + (tok0 + (key0 + r - plen)) * a.ldqkv + (which ? v_off : k_off) + kvh * DH + c * 8;
-          const int64_t step = (int64_t)RPP * a.ldqkv;
-#pragma unroll 4
-          for (; r < nt; r += RPP, src += step) cp_async16(dst + box + swz(r, c & 7), src);
-#pragma unroll 4
-          for (; r < KEY_BLOCK; r += RPP) *reinterpret_cast<uint4*>(dst + box + swz(r, c & 7)) = make_uint4(0, 0, 0, 0);
+            for (int j = 0; j < DH / 64; ++j)
+              ptx::tma_load_3d(dst + j * (KEY_BLOCK * 128), pm, j * 64, blk * KEY_BLOCK, plane, &full_bar[s]);
+          } else {
+            if (!waited) { ptx::pdl_wait_prior_grids(); waited = true; }  // only the suffix rows depend on the preceding grid
+            const int rowg = (int)tok0 + (blk - npb) * KEY_BLOCK;
+#pragma unroll
+            for (int j = 0; j < DH / 64; ++j)
+              ptx::tma_load_2d(dst + j * (KEY_BLOCK * 128), &map_sfx, (which ? v_off : k_off) + kvh * DH + j * 64, rowg, &full_bar[s]);
+          }
+          if (dbg && tid == 128 && item == (int)blockIdx.x && i < 2) dbg[3 + i] = ptx::globaltimer_ns();
+          if (dlog && tid == 128 && item == 0 && i < 32) dlog[i * 4 + 0] = ptx::globaltimer_ns();
         }
-        cp_async_commit();
-        cp_async_wait_all();
-        ptx::fence_proxy_async();
-        ptx::mbar_arrive(&full_bar[s]);
-        if (dbg && tid == 128 && item == (int)blockIdx.x && i < 2) dbg[3 + i] = ptx::globaltimer_ns();
-        if (dlog && tid == 128 && item == 0 && i < 32) dlog[i * 4 + 0] = ptx::globaltimer_ns();
       }
+      ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+      if (!waited && PARTIAL) { ptx::pdl_wait_prior_grids(); waited = true; }  // (before this warp writes partial outputs)
       // Their loads done, the loader warps help to stage a key split's unnormalised output: warp w can read the same
       // TMEM lanes as softmax warp w - 4, and takes the upper half of the channels.
       if (PARTIAL && nb > 0 && ok) {
@@ -329,19 +317,21 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
         if (lane == 0) ptx::mbar_arrive(&s_empty[s]);
         // block maximum of the raw scores (the scale is positive, so it commutes with max); only the last
         // block of a key list can hold columns outside it, which are masked to -inf
-        const int key0 = (kb0 + i) * KEY_BLOCK;
-        if (key0 + KEY_BLOCK > total) {
+        // keys of this block that exist: a prefix block ends at prefix_len, a suffix block at the token count
+        const int blk = kb0 + i;
+        const int nvalid = blk < npb ? min(KEY_BLOCK, plen - blk * KEY_BLOCK) : min(KEY_BLOCK, a.n_tokens - (blk - npb) * KEY_BLOCK);
+        if (nvalid < KEY_BLOCK) {
 #pragma unroll
           for (int j = 0; j < 64; ++j)
-            if (key0 + j >= total) sc[j] = -INFINITY;
+            if (j >= nvalid) sc[j] = -INFINITY;
         }
-        // variant: the state token's rows (token 0 of the request: rows 0 .. G-1 of row tile 0) see the prefix and
+        // variant: the state token's rows (token 0 of the request: rows 0 .. G-1 of row tile 0) see, of the suffix,
         // the state token's own key only
-        const bool state_row = a.state_mask && rt * TC_ROWS + row < G;
-        if (state_row && key0 + KEY_BLOCK > plen + 1) {
+        if (a.state_mask && rt * TC_ROWS + row < G && blk >= npb) {
+          const int first = (blk - npb) * KEY_BLOCK;
 #pragma unroll
           for (int j = 0; j < 64; ++j)
-            if (key0 + j > plen) sc[j] = -INFINITY;
+            if (first + j > 0) sc[j] = -INFINITY;
         }
         // (four independent chains: a single thread per scheduler cannot hide the latency of one long chain)
         float mx[4] = {sc[0], sc[1], sc[2], sc[3]};

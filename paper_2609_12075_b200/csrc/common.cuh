@@ -1,5 +1,6 @@
 // Shared declarations of the ADiT library: element types, small device helpers, epilogue ids.
 #pragma once
+#include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -44,6 +45,14 @@ struct EpiArgs {
 struct PrefixTable {
   const void* kv[64];
   int32_t len[64];
+};
+
+// Per-call tensor maps of the requests' prefix caches for the tensor-core attention kernel: request b's cache seen
+// as a 3-D tensor (channel, row, plane = (layer, K|V, kv head)) whose row extent is prefix_len[b], so that rows at or
+// beyond it are never read (the copy engine writes zeros for them).  Written to device memory by a small kernel
+// from its by-value parameter, like the call descriptor.
+struct KvMaps {
+  alignas(64) CUtensorMap pk[64];
 };
 
 // Everything that changes from one adit_denoise call to the next.  The kernels of the captured launch

@@ -86,6 +86,7 @@ struct GemmLv {
 
 struct LoopParams {
   alignas(64) CUtensorMap pk[MAXB];  // per request: prefix cache as (channel, row < prefix_len, plane)
+  alignas(64) CUtensorMap kv2d;      // this step's K/V rows of the qkv workspace, row extent = the call's token count
   const CUtensorMap* maps;           // device array, see MAP_*
   int plen[MAXB];
   GemmLv g[G_COUNT];
@@ -335,11 +336,11 @@ __device__ void role_weights(const Ctx& c) {
             if (!bwait(c, &ms->k_empty[st], par ^ 1u)) { ok = false; break; }
             ptx::mbar_arrive_expect_tx(&ms->k_full[st], KVB);
             for (int j = 0; j < DH / 64; ++j)
-              ptx::tma_load_2d(kd + j * (attn::KEY_BLOCK * 128), &p.maps[MAP_KV2D], k_off + a.kvh * DH + j * 64, row, &ms->k_full[st]);
+              ptx::tma_load_2d(kd + j * (attn::KEY_BLOCK * 128), &p.kv2d, k_off + a.kvh * DH + j * 64, row, &ms->k_full[st]);
             if (!bwait(c, &ms->v_empty[st], par ^ 1u)) { ok = false; break; }
             ptx::mbar_arrive_expect_tx(&ms->v_full[st], KVB);
             for (int j = 0; j < DH / 64; ++j)
-              ptx::tma_load_2d(vd + j * (attn::KEY_BLOCK * 128), &p.maps[MAP_KV2D], v_off + a.kvh * DH + j * 64, row, &ms->v_full[st]);
+              ptx::tma_load_2d(vd + j * (attn::KEY_BLOCK * 128), &p.kv2d, v_off + a.kvh * DH + j * 64, row, &ms->v_full[st]);
           }
         }
         // no weight may land in these bytes before the unit is over

@@ -69,6 +69,12 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, uint64
 __device__ __forceinline__ void prefetch_tensormap(const CUtensorMap* m) {
   asm volatile("prefetch.tensormap [%0];" ::"l"(m) : "memory");
 }
+// Tensor maps that a kernel wrote to global memory: the writer releases, the thread that is going to use the map
+// for a copy acquires (the copy engine reads maps through a cache of its own).
+__device__ __forceinline__ void tensormap_release() { asm volatile("fence.proxy.tensormap::generic.release.gpu;" ::: "memory"); }
+__device__ __forceinline__ void tensormap_acquire(const CUtensorMap* m) {
+  asm volatile("fence.proxy.tensormap::generic.acquire.gpu [%0], 128;" ::"l"(m) : "memory");
+}
 // 2-D tiled load global -> shared, completion counted in bytes on `bar`.  x = innermost (element)
 // coordinate, which must be a multiple of 16 bytes worth of elements; y = row.
 __device__ __forceinline__ void tma_load_2d(void* smem_dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
