@@ -260,7 +260,8 @@ def run_ours(args):
     base = WORKLOADS[args.workload]()
     cfg = base.cfg
     weights = W.make_weights(cfg, base.seed)
-    flags = (adit.FLAG_NO_GRAPH if args.no_graph else 0) | (adit.FLAG_PERSISTENT_LOOP if args.persistent else 0)
+    flags = (adit.FLAG_NO_GRAPH if args.no_graph else 0) | (adit.FLAG_PERSISTENT_LOOP if args.persistent else 0) | \
+        (adit.FLAG_ONE_SM_GEMM if args.one_sm_gemm else 0)
     eng = adit.ADiT(cfg, max_batch=base.batch, max_prefix_len=base.max_prefix_len, device=local, flags=flags)
     eng.load_weights(weights)
     sets = make_sets(adit, base, n_sets, rank, local, dev, torch)
@@ -693,6 +694,7 @@ def main():
     ap.add_argument("--no-trace", action="store_true", help="skip the in-situ timeline of one call")
     ap.add_argument("--no-extra", action="store_true", help="skip the brief runs of the other batch sizes (c3, c4)")
     ap.add_argument("--no-graph", action="store_true", help="enqueue kernels one by one (ADIT_FLAG_NO_GRAPH): for profilers")
+    ap.add_argument("--one-sm-gemm", action="store_true", help="projections on the one-SM kernel at every batch size (ADIT_FLAG_ONE_SM_GEMM): comparison")
     ap.add_argument("--persistent", action="store_true", help="small batches as one persistent kernel (ADIT_FLAG_PERSISTENT_LOOP)")
     ap.add_argument("--latency-calls", type=int, default=None, help="calls sampled for p50/p99 (default 1000 at batch 1)")
     ap.add_argument("--latency-seconds", type=float, default=12.0, help="wall budget of the latency sampling")

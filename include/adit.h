@@ -58,6 +58,7 @@ typedef enum {
 #define ADIT_FLAG_STATE_BLOCK_MASK 32 /* model variant: the state token attends to the prefix and itself only, not to the action tokens */
 #define ADIT_FLAG_SUFFIX_ROPE 64      /* model variant: rotary embedding (pairs j, j + head_dim/2; base 10000) on the suffix queries
                                          and keys at positions prefix_len[b] + index in the suffix; prefix keys are used as given */
+#define ADIT_FLAG_ONE_SM_GEMM 128     /* projections on the one-SM kernel at every batch size (comparison aid; large batches otherwise use two-SM products) */
 #define ADIT_FLAG_PERSISTENT_LOOP 16  /* small batches run as one persistent kernel instead of a kernel per phase (see adit_uses_persistent_loop) */
 
 typedef struct adit_handle adit_handle; /* opaque; owns packed weights and a workspace on one device */
@@ -253,9 +254,10 @@ int64_t adit_debug_copy(adit_handle* h, const char* name, void* host_dst, size_t
 /*
  * adit_debug_gemm: run the tensor-core projection kernel on its own (test aid): out[n_tok, n_feat]
  * (fp32, device) = A[n_tok, k] W[n_feat, k]^T with bf16 device operands, k a multiple of 64;
- * splits = 0 lets the library choose the k-split, sm_budget as in adit_denoise.  Synchronises the
+ * splits = 0 lets the library choose the k-split, splits = -2 selects the two-SM kernel (pairs of
+ * thread blocks, 256 features x tile_tokens per pair), sm_budget as in adit_denoise.  Synchronises the
  * stream.  Returns a negative status, or a positive plan code splits * 1e6 + tile_tokens * 1e3 +
- * pipeline stages.  The paper has no counterpart.
+ * pipeline stages (splits reads 9 for the two-SM kernel).  The paper has no counterpart.
  */
 int adit_debug_gemm(int device, int n_tok, int n_feat, int k, const void* a_bf16, const void* w_bf16,
                     float* out_f32, int splits, int sm_budget, void* stream);
@@ -348,10 +350,12 @@ int adit_debug_stream_read(int device, size_t bytes, int sm_count, int iters, do
  * stand-in for the VLM stage that shares the GPU with the ADiT stream (section 4.1.2: the VLM
  * stream is restricted to a number of SMs so that the ADiT kernels always find free ones).
  * create allocates the operands (deterministic fill); launch enqueues `iters` repetitions on
- * `stream` using at most `sm_count` SMs (<= 0: all).
+ * `stream` using at most `sm_count` SMs (<= 0: all).  create_kind chooses the kernel: 0 = the one-SM
+ * projection kernel (what create uses), 1 = the two-SM kernel (pairs of thread blocks).
  */
 typedef struct adit_bg_gemm adit_bg_gemm;
 int adit_bg_gemm_create(int device, int m, int n, int k, adit_bg_gemm** out);
+int adit_bg_gemm_create_kind(int device, int m, int n, int k, int kind, adit_bg_gemm** out);
 int adit_bg_gemm_launch(adit_bg_gemm* g, int iters, int sm_count, void* stream);
 int adit_bg_gemm_destroy(adit_bg_gemm* g);
 

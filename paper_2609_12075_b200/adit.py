@@ -22,13 +22,13 @@ lib = C.CDLL(_LIB_PATH)
 OK, E_INVALID, E_CAPACITY, E_NOT_LOADED, E_UNSUPPORTED, E_CUDA, E_TIMEOUT = 0, -1, -2, -3, -4, -5, -6
 DTYPE_FP32, DTYPE_BF16 = 0, 1
 FLAG_REFERENCE_KERNELS, FLAG_NO_GRAPH, FLAG_NO_PDL, FLAG_MMA_SYNC_ATTENTION, FLAG_PERSISTENT_LOOP = 1, 2, 4, 8, 16
-FLAG_STATE_BLOCK_MASK, FLAG_SUFFIX_ROPE = 32, 64
+FLAG_STATE_BLOCK_MASK, FLAG_SUFFIX_ROPE, FLAG_ONE_SM_GEMM = 32, 64, 128
 MAX_BATCH, MAX_STEPS = 64, 64
 
 EXPORTS = ["adit_create", "adit_load_weights", "adit_denoise", "adit_denoise_host", "adit_destroy",
            "adit_poll_status", "adit_last_cuda_error", "adit_kernel_launches", "adit_strerror",
            "adit_debug_copy", "adit_debug_gemm", "adit_debug_plan", "adit_debug_gemm_stamps", "adit_debug_attention", "adit_attention_static", "adit_profile_enable", "adit_profile_read", "adit_profile_class_name", "adit_trace_enable", "adit_trace_read",
-           "adit_bg_gemm_create", "adit_bg_gemm_launch", "adit_bg_gemm_destroy",
+           "adit_bg_gemm_create", "adit_bg_gemm_create_kind", "adit_bg_gemm_launch", "adit_bg_gemm_destroy",
            "adit_debug_stream_read", "adit_attention_static_status", "adit_debug_stamps_selected",
            "adit_clear_status", "adit_uses_persistent_loop", "adit_debug_wait_limit", "adit_loop_trace_read"]
 
@@ -86,6 +86,7 @@ lib.adit_debug_wait_limit.argtypes = [C.c_void_p, C.c_int, C.c_int]
 lib.adit_loop_trace_read.argtypes = [C.c_void_p, C.POINTER(C.c_int64), C.c_int64]
 lib.adit_loop_trace_read.restype = C.c_int64
 lib.adit_bg_gemm_create.argtypes = [C.c_int, C.c_int, C.c_int, C.c_int, C.POINTER(C.c_void_p)]
+lib.adit_bg_gemm_create_kind.argtypes = [C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, C.POINTER(C.c_void_p)]
 lib.adit_bg_gemm_launch.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_void_p]
 lib.adit_bg_gemm_destroy.argtypes = [C.c_void_p]
 
@@ -272,9 +273,9 @@ def upload_prefix_kv(wl: W.Workload, device: int = 0) -> List:
 class BackgroundGemm:
     """Looping bf16 GEMM on a capped number of SMs (the VLM-stage stand-in on the other stream)."""
 
-    def __init__(self, m: int, n: int, k: int, device: int = 0):
+    def __init__(self, m: int, n: int, k: int, device: int = 0, two_sm: bool = False):
         self._g = C.c_void_p()
-        rc = lib.adit_bg_gemm_create(device, m, n, k, C.byref(self._g))
+        rc = lib.adit_bg_gemm_create_kind(device, m, n, k, 1 if two_sm else 0, C.byref(self._g))
         if rc != OK:
             self._g = C.c_void_p()
             raise AditError(rc)

@@ -746,13 +746,14 @@ static int enqueue_tc(adit_handle* h, int B, int K, int G, cudaStream_t st) {
   h->trace_off = 0;
   auto cap = [&](int64_t blocks) { return (int)((capped && blocks > G) ? G : blocks); };
   // plans and activation descriptors for this batch size
-  tc::GemmPlan p_e2 = tc::plan_gemm(Ma, D, D, false, SM, true),
-               p_qkv = tc::plan_gemm(M, QKV, D, false, SM, true), p_o = tc::plan_gemm(M, D, Q, false, SM, true),
-               p_gu = tc::plan_gemm(M, F, D, true, SM, true), p_d = tc::plan_gemm(M, D, F, false, SM, true);
+  const bool two_sm = !(c.flags & ADIT_FLAG_ONE_SM_GEMM);
+  tc::GemmPlan p_e2 = tc::plan_projection(Ma, D, D, false, SM, two_sm),
+               p_qkv = tc::plan_projection(M, QKV, D, false, SM, two_sm), p_o = tc::plan_projection(M, D, Q, false, SM, two_sm),
+               p_gu = tc::plan_projection(M, F, D, true, SM, two_sm), p_d = tc::plan_projection(M, D, F, false, SM, two_sm);
   CUtensorMap a_e2, a_qkv, a_o, a_gu, a_d;
-  bool ok = tc::make_map_bf16(&a_e2, h->ez, Max, D, p_e2.tile_tok) &&
-            tc::make_map_bf16(&a_qkv, h->hb, Mx, D, p_qkv.tile_tok) && tc::make_map_bf16(&a_o, h->att, Mx, Q, p_o.tile_tok) &&
-            tc::make_map_bf16(&a_gu, h->hb, Mx, D, p_gu.tile_tok) && tc::make_map_bf16(&a_d, h->mlp, Mx, F, p_d.tile_tok);
+  bool ok = tc::make_map_bf16(&a_e2, h->ez, Max, D, tc::token_box_rows(p_e2)) &&
+            tc::make_map_bf16(&a_qkv, h->hb, Mx, D, tc::token_box_rows(p_qkv)) && tc::make_map_bf16(&a_o, h->att, Mx, Q, tc::token_box_rows(p_o)) &&
+            tc::make_map_bf16(&a_gu, h->hb, Mx, D, tc::token_box_rows(p_gu)) && tc::make_map_bf16(&a_d, h->mlp, Mx, F, tc::token_box_rows(p_d));
   if (!ok) return ADIT_E_CUDA;
 
   auto gemm = [&](int cls, const CUtensorMap& mw, const CUtensorMap& ma, const tc::GemmPlan& p, bool dual, int n_tok,
@@ -1546,9 +1547,10 @@ extern "C" int adit_debug_gemm(int device, int n_tok, int n_feat, int k, const v
   if (prop.major != 10) return ADIT_E_UNSUPPORTED;
   if (tc::ensure_smem_attr() != cudaSuccess) return ADIT_E_CUDA;
   const int SM = prop.multiProcessorCount;
-  tc::GemmPlan p = tc::plan_gemm(n_tok, n_feat, k, false, SM, true, splits);
+  if (splits == -2 && SM < 2) return ADIT_E_UNSUPPORTED;
+  tc::GemmPlan p = splits == -2 ? tc::plan_gemm_pair(n_tok, n_feat, k, false, SM) : tc::plan_gemm(n_tok, n_feat, k, false, SM, true, splits);
   CUtensorMap mw, ma;
-  if (!tc::make_map_bf16(&mw, w_bf16, n_feat, k, tc::TILE_F) || !tc::make_map_bf16(&ma, a_bf16, n_tok, k, p.tile_tok))
+  if (!tc::make_map_bf16(&mw, w_bf16, n_feat, k, tc::TILE_F) || !tc::make_map_bf16(&ma, a_bf16, n_tok, k, tc::token_box_rows(p)))
     return ADIT_E_CUDA;
   int* status = nullptr;
   float* tmp = nullptr;  // the kernel stores whole token tiles: give it the padding rows the library's buffers have
@@ -1572,7 +1574,7 @@ extern "C" int adit_debug_gemm(int device, int n_tok, int n_feat, int k, const v
     cudaGetLastError();
     return ADIT_E_CUDA;
   }
-  return hs ? hs : (p.splits * 1000000 + p.tile_tok * 1000 + p.stages);  // plan, for the test's information
+  return hs ? hs : ((p.pair ? 9 : p.splits) * 1000000 + p.tile_tok * 1000 + p.stages);  // plan, for the test's information (9 = two-SM kernel)
 }
 
 
@@ -1641,7 +1643,11 @@ __global__ void bg_fill_kernel(bf16* __restrict__ p, int64_t n, uint32_t seed) {
 }
 
 extern "C" int adit_bg_gemm_create(int device, int m, int n, int k, adit_bg_gemm** out) {
-  if (!out || m < 1 || n < 1 || k < 64 || (k % 64)) return ADIT_E_INVALID;
+  return adit_bg_gemm_create_kind(device, m, n, k, 0, out);
+}
+
+extern "C" int adit_bg_gemm_create_kind(int device, int m, int n, int k, int kind, adit_bg_gemm** out) {
+  if (!out || m < 1 || n < 1 || k < 64 || (k % 64) || kind < 0 || kind > 1) return ADIT_E_INVALID;
   if (cudaSetDevice(device) != cudaSuccess) return ADIT_E_CUDA;
   cudaDeviceProp prop;
   if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return ADIT_E_CUDA;
@@ -1651,7 +1657,8 @@ extern "C" int adit_bg_gemm_create(int device, int m, int n, int k, adit_bg_gemm
   if (!g) return ADIT_E_INVALID;
   g->device = device; g->m = m; g->n = n; g->k = k; g->sm_count = prop.multiProcessorCount;
   g->a = g->b = g->c = nullptr; g->status = nullptr;
-  g->plan = tc::plan_gemm(m, n, k, false, g->sm_count, false);
+  if (kind == 1 && g->sm_count < 2) { delete g; return ADIT_E_UNSUPPORTED; }
+  g->plan = kind == 1 ? tc::plan_gemm_pair(m, n, k, false, g->sm_count) : tc::plan_gemm(m, n, k, false, g->sm_count, false);
   const size_t rows_c = (size_t)g->plan.n_ttiles * g->plan.tile_tok;  // whole token tiles are stored
   bool ok = cudaMalloc(&g->a, (size_t)m * k * 2) == cudaSuccess && cudaMalloc(&g->b, (size_t)n * k * 2) == cudaSuccess &&
             cudaMalloc(&g->c, rows_c * n * 2) == cudaSuccess && cudaMalloc((void**)&g->status, 4) == cudaSuccess;
@@ -1659,7 +1666,7 @@ extern "C" int adit_bg_gemm_create(int device, int m, int n, int k, adit_bg_gemm
     cudaMemset(g->status, 0, 4);
     bg_fill_kernel<<<1024, 256>>>((bf16*)g->a, (int64_t)m * k, 1u);
     bg_fill_kernel<<<1024, 256>>>((bf16*)g->b, (int64_t)n * k, 2u);
-    ok = cudaDeviceSynchronize() == cudaSuccess && tc::make_map_bf16(&g->map_a, g->a, m, k, g->plan.tile_tok) &&
+    ok = cudaDeviceSynchronize() == cudaSuccess && tc::make_map_bf16(&g->map_a, g->a, m, k, tc::token_box_rows(g->plan)) &&
          tc::make_map_bf16(&g->map_b, g->b, n, k, tc::TILE_F);
   }
   if (!ok) {

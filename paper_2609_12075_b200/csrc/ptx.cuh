@@ -208,6 +208,243 @@ __device__ __forceinline__ uint32_t idesc_bf16_f32(int m, int n) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
 }
 
+// ---- one k-block (64 deep = four products of 16) issued as a single instruction sequence ------------------------
+// The issuing thread has nothing to hide its own instruction latencies behind, and a product should leave it every
+// 60-130 cycles: descriptors are therefore kept as 32-bit halves (only the low half, which holds the address, changes
+// from product to product: + 2 per 32 bytes along k) and the four products of a k-block are one asm block.
+// `lo` halves: see smem_desc_lo; `hi`: smem_desc_hi_sw128 (the same for every K-major 128-byte-swizzled operand).
+__device__ __forceinline__ uint32_t smem_desc_lo(uint32_t smem_addr) { return ((smem_addr & 0x3FFFF) >> 4) | (1u << 16); }
+__device__ __forceinline__ uint32_t smem_desc_hi_sw128() { return (uint32_t)(1024 >> 4) | (1u << 14) | (2u << 29); }
+#define ADIT_UMMA_KBLOCK(NAME, GROUP)                                                                              \
+  __device__ __forceinline__ void NAME(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t hi, uint32_t idesc, \
+                                       uint32_t acc_first) {                                                       \
+    asm volatile(                                                                                                  \
+        "{\n\t.reg .pred p, q;\n\t.reg .b64 a, b;\n\t.reg .b32 al, bl;\n\t"                                        \
+        "setp.ne.b32 p, %5, 0;\n\t"                                                                                \
+        "setp.eq.b32 q, 0, 0;\n\t"                                                                                 \
+        "mov.b64 a, {%1, %3};\n\tmov.b64 b, {%2, %3};\n\t"                                                         \
+        "tcgen05.mma.cta_group::" GROUP ".kind::f16 [%0], a, b, %4, p;\n\t"                                        \
+        "add.u32 al, %1, 2;\n\tadd.u32 bl, %2, 2;\n\tmov.b64 a, {al, %3};\n\tmov.b64 b, {bl, %3};\n\t"             \
+        "tcgen05.mma.cta_group::" GROUP ".kind::f16 [%0], a, b, %4, q;\n\t"                                        \
+        "add.u32 al, %1, 4;\n\tadd.u32 bl, %2, 4;\n\tmov.b64 a, {al, %3};\n\tmov.b64 b, {bl, %3};\n\t"             \
+        "tcgen05.mma.cta_group::" GROUP ".kind::f16 [%0], a, b, %4, q;\n\t"                                        \
+        "add.u32 al, %1, 6;\n\tadd.u32 bl, %2, 6;\n\tmov.b64 a, {al, %3};\n\tmov.b64 b, {bl, %3};\n\t"             \
+        "tcgen05.mma.cta_group::" GROUP ".kind::f16 [%0], a, b, %4, q;\n\t}" ::"r"(d_tmem),                        \
+        "r"(a_lo), "r"(b_lo), "r"(hi), "r"(idesc), "r"(acc_first)                                                  \
+        : "memory");                                                                                               \
+  }
+ADIT_UMMA_KBLOCK(umma_kblock_f16, "1")
+ADIT_UMMA_KBLOCK(umma_kblock_f16_pair, "2")
+#undef ADIT_UMMA_KBLOCK
+// The same for a gate/up pair: two accumulators (d_tmem, d_tmem2), two weight operands, one token operand.
+#define ADIT_UMMA_KBLOCK2(NAME, GROUP)                                                                             \
+  __device__ __forceinline__ void NAME(uint32_t d_tmem, uint32_t d_tmem2, uint32_t a_lo, uint32_t a2_lo,           \
+                                       uint32_t b_lo, uint32_t hi, uint32_t idesc, uint32_t acc_first) {           \
+    asm volatile(                                                                                                  \
+        "{\n\t.reg .pred p, q;\n\t.reg .b64 a, a2, b;\n\t.reg .b32 al, a2l, bl;\n\t"                               \
+        "setp.ne.b32 p, %7, 0;\n\t"                                                                                \
+        "setp.eq.b32 q, 0, 0;\n\t"                                                                                 \
+        "mov.b64 a, {%2, %5};\n\tmov.b64 a2, {%3, %5};\n\tmov.b64 b, {%4, %5};\n\t"                                \
+        "tcgen05.mma.cta_group::" GROUP ".kind::f16 [%0], a, b, %6, p;\n\t"                                        \
+        "tcgen05.mma.cta_group::" GROUP ".kind::f16 [%1], a2, b, %6, p;\n\t"                                       \
+        "add.u32 al, %2, 2;\n\tadd.u32 a2l, %3, 2;\n\tadd.u32 bl, %4, 2;\n\t"                                      \
+        "mov.b64 a, {al, %5};\n\tmov.b64 a2, {a2l, %5};\n\tmov.b64 b, {bl, %5};\n\t"                               \
+        "tcgen05.mma.cta_group::" GROUP ".kind::f16 [%0], a, b, %6, q;\n\t"                                        \
+        "tcgen05.mma.cta_group::" GROUP ".kind::f16 [%1], a2, b, %6, q;\n\t"                                       \
+        "add.u32 al, %2, 4;\n\tadd.u32 a2l, %3, 4;\n\tadd.u32 bl, %4, 4;\n\t"                                      \
+        "mov.b64 a, {al, %5};\n\tmov.b64 a2, {a2l, %5};\n\tmov.b64 b, {bl, %5};\n\t"                               \
+        "tcgen05.mma.cta_group::" GROUP ".kind::f16 [%0], a, b, %6, q;\n\t"                                        \
+        "tcgen05.mma.cta_group::" GROUP ".kind::f16 [%1], a2, b, %6, q;\n\t"                                       \
+        "add.u32 al, %2, 6;\n\tadd.u32 a2l, %3, 6;\n\tadd.u32 bl, %4, 6;\n\t"                                      \
+        "mov.b64 a, {al, %5};\n\tmov.b64 a2, {a2l, %5};\n\tmov.b64 b, {bl, %5};\n\t"                               \
+        "tcgen05.mma.cta_group::" GROUP ".kind::f16 [%0], a, b, %6, q;\n\t"                                        \
+        "tcgen05.mma.cta_group::" GROUP ".kind::f16 [%1], a2, b, %6, q;\n\t}" ::"r"(d_tmem),                       \
+        "r"(d_tmem2), "r"(a_lo), "r"(a2_lo), "r"(b_lo), "r"(hi), "r"(idesc), "r"(acc_first)                        \
+        : "memory");                                                                                               \
+  }
+ADIT_UMMA_KBLOCK2(umma_kblock2_f16, "1")
+ADIT_UMMA_KBLOCK2(umma_kblock2_f16_pair, "2")
+#undef ADIT_UMMA_KBLOCK2
+
+// A whole step of the issuing thread's k loop as one instruction sequence: test the NEXT stage's "filled" barrier
+// (result wanted one step later), issue this k-block's four products (eight for a gate/up pair), commit them to this
+// stage's "free" barrier, and only then read the test's result - so that the barrier test's latency is hidden behind
+// the products' issue instead of stalling the (in-order) thread.  Returns whether the next stage is already filled.
+// The two-SM form commits to the same barrier offset in both blocks of the pair.  Barriers are given as 32-bit
+// shared-memory addresses (smem_u32), which the caller keeps in registers: every instruction of this thread counts.
+#define ADIT_COMMIT_1 "tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%7];\n\t"
+#define ADIT_COMMIT_2 "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%7], m;\n\t"
+#define ADIT_UMMA_STEP(NAME, GROUP, COMMIT)                                                                          \
+  __device__ __forceinline__ bool NAME(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t hi, uint32_t idesc,   \
+                                       uint32_t acc_first, uint32_t free_bar, uint32_t next_full, uint32_t parity) { \
+    uint32_t ready;                                                                                                  \
+    asm volatile(                                                                                                    \
+        "{\n\t.reg .pred p, q, r;\n\t.reg .b64 a, b;\n\t.reg .b32 al, bl;\n\t.reg .b16 m;\n\tmov.b16 m, 3;\n\t"     \
+        "mbarrier.test_wait.parity.shared::cta.b64 r, [%8], %9;\n\t"                                                 \
+        "setp.ne.b32 p, %6, 0;\n\t"                                                                                  \
+        "setp.eq.b32 q, 0, 0;\n\t"                                                                                   \
+        "mov.b64 a, {%2, %4};\n\tmov.b64 b, {%3, %4};\n\t"                                                           \
+        "tcgen05.mma.cta_group::" GROUP ".kind::f16 [%1], a, b, %5, p;\n\t"                                          \
+        "add.u32 al, %2, 2;\n\tadd.u32 bl, %3, 2;\n\tmov.b64 a, {al, %4};\n\tmov.b64 b, {bl, %4};\n\t"               \
+        "tcgen05.mma.cta_group::" GROUP ".kind::f16 [%1], a, b, %5, q;\n\t"                                          \
+        "add.u32 al, %2, 4;\n\tadd.u32 bl, %3, 4;\n\tmov.b64 a, {al, %4};\n\tmov.b64 b, {bl, %4};\n\t"               \
+        "tcgen05.mma.cta_group::" GROUP ".kind::f16 [%1], a, b, %5, q;\n\t"                                          \
+        "add.u32 al, %2, 6;\n\tadd.u32 bl, %3, 6;\n\tmov.b64 a, {al, %4};\n\tmov.b64 b, {bl, %4};\n\t"               \
+        "tcgen05.mma.cta_group::" GROUP ".kind::f16 [%1], a, b, %5, q;\n\t" COMMIT                                   \
+        "selp.u32 %0, 1, 0, r;\n\t}"                                                                                 \
+        : "=r"(ready)                                                                                                \
+        : "r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(hi), "r"(idesc), "r"(acc_first), "r"(free_bar),                     \
+          "r"(next_full), "r"(parity)                                                                      \
+        : "memory");                                                                                                 \
+    return ready != 0;                                                                                               \
+  }
+ADIT_UMMA_STEP(umma_step_f16, "1", ADIT_COMMIT_1)
+ADIT_UMMA_STEP(umma_step_f16_pair, "2", ADIT_COMMIT_2)
+#undef ADIT_UMMA_STEP
+#undef ADIT_COMMIT_1
+#undef ADIT_COMMIT_2
+#define ADIT_COMMIT_1 "tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%9];\n\t"
+#define ADIT_COMMIT_2 "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%9], m;\n\t"
+#define ADIT_UMMA_STEP2(NAME, GROUP, COMMIT)                                                                         \
+  __device__ __forceinline__ bool NAME(uint32_t d_tmem, uint32_t d_tmem2, uint32_t a_lo, uint32_t a2_lo, uint32_t b_lo, \
+                                       uint32_t hi, uint32_t idesc, uint32_t acc_first, uint32_t free_bar,           \
+                                       uint32_t next_full, uint32_t parity) {                                       \
+    uint32_t ready;                                                                                                  \
+    asm volatile(                                                                                                    \
+        "{\n\t.reg .pred p, q, r;\n\t.reg .b64 a, a2, b;\n\t.reg .b32 al, a2l, bl;\n\t.reg .b16 m;\n\tmov.b16 m, 3;\n\t" \
+        "mbarrier.test_wait.parity.shared::cta.b64 r, [%10], %11;\n\t"                                               \
+        "setp.ne.b32 p, %8, 0;\n\t"                                                                                  \
+        "setp.eq.b32 q, 0, 0;\n\t"                                                                                   \
+        "mov.b64 a, {%3, %6};\n\tmov.b64 a2, {%4, %6};\n\tmov.b64 b, {%5, %6};\n\t"                                  \
+        "tcgen05.mma.cta_group::" GROUP ".kind::f16 [%1], a, b, %7, p;\n\t"                                          \
+        "tcgen05.mma.cta_group::" GROUP ".kind::f16 [%2], a2, b, %7, p;\n\t"                                         \
+        "add.u32 al, %3, 2;\n\tadd.u32 a2l, %4, 2;\n\tadd.u32 bl, %5, 2;\n\t"                                        \
+        "mov.b64 a, {al, %6};\n\tmov.b64 a2, {a2l, %6};\n\tmov.b64 b, {bl, %6};\n\t"                                 \
+        "tcgen05.mma.cta_group::" GROUP ".kind::f16 [%1], a, b, %7, q;\n\t"                                          \
+        "tcgen05.mma.cta_group::" GROUP ".kind::f16 [%2], a2, b, %7, q;\n\t"                                         \
+        "add.u32 al, %3, 4;\n\tadd.u32 a2l, %4, 4;\n\tadd.u32 bl, %5, 4;\n\t"                                        \
+        "mov.b64 a, {al, %6};\n\tmov.b64 a2, {a2l, %6};\n\tmov.b64 b, {bl, %6};\n\t"                                 \
+        "tcgen05.mma.cta_group::" GROUP ".kind::f16 [%1], a, b, %7, q;\n\t"                                          \
+        "tcgen05.mma.cta_group::" GROUP ".kind::f16 [%2], a2, b, %7, q;\n\t"                                         \
+        "add.u32 al, %3, 6;\n\tadd.u32 a2l, %4, 6;\n\tadd.u32 bl, %5, 6;\n\t"                                        \
+        "mov.b64 a, {al, %6};\n\tmov.b64 a2, {a2l, %6};\n\tmov.b64 b, {bl, %6};\n\t"                                 \
+        "tcgen05.mma.cta_group::" GROUP ".kind::f16 [%1], a, b, %7, q;\n\t"                                          \
+        "tcgen05.mma.cta_group::" GROUP ".kind::f16 [%2], a2, b, %7, q;\n\t" COMMIT                                  \
+        "selp.u32 %0, 1, 0, r;\n\t}"                                                                                 \
+        : "=r"(ready)                                                                                                \
+        : "r"(d_tmem), "r"(d_tmem2), "r"(a_lo), "r"(a2_lo), "r"(b_lo), "r"(hi), "r"(idesc), "r"(acc_first),          \
+          "r"(free_bar), "r"(next_full), "r"(parity)                                             \
+        : "memory");                                                                                                 \
+    return ready != 0;                                                                                               \
+  }
+ADIT_UMMA_STEP2(umma_step2_f16, "1", ADIT_COMMIT_1)
+ADIT_UMMA_STEP2(umma_step2_f16_pair, "2", ADIT_COMMIT_2)
+#undef ADIT_UMMA_STEP2
+#undef ADIT_COMMIT_1
+#undef ADIT_COMMIT_2
+
+__device__ __forceinline__ bool mbar_test_wait_addr(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait for a thread that must react at once (the product issuer): non-blocking tests in a tight loop for
+// about ten microseconds before the clocked, slower loop of mbar_wait takes over.
+__device__ __forceinline__ bool mbar_wait_hot(uint64_t* bar, uint32_t parity) {
+#pragma unroll 1
+  for (int i = 0; i < 2048; ++i)
+    if (mbar_test_wait(bar, parity)) return true;
+  return mbar_wait(bar, parity);
+}
+// hot_polls: non-blocking tests before the clocked loop (0 = go to the clock at once: its read takes a few hundred
+// nanoseconds, which is a welcome back-off where the data is known to be far away)
+__device__ __noinline__ bool mbar_wait_hot_addr(uint32_t bar, uint32_t parity, int hot_polls = 2048) {  // (the slow path: kept out of line)
+#pragma unroll 1
+  for (int i = 0; i < hot_polls; ++i)
+    if (mbar_test_wait_addr(bar, parity)) return true;
+  const uint64_t t0 = globaltimer_ns();
+  for (;;) {
+#pragma unroll 1
+    for (int i = 0; i < 1024; ++i)
+      if (mbar_test_wait_addr(bar, parity)) return true;
+    if (globaltimer_ns() - t0 > 2000000000ull) return false;
+  }
+}
+
+// ---- the two-SM forms (cta_group::2): a pair of blocks of one cluster (ranks 2i, 2i + 1) works on one product ------
+// Every tcgen05 instruction of a kernel names the same cta_group, so a kernel uses either these or the forms above.
+// Allocation and release are executed by one warp of each block of the pair; both get the same column range.
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t* smem_result, uint32_t ncols) {  // whole warp
+  asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(smem_result)),
+               "r"(ncols)
+               : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish_pair() {  // whole warp
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t ncols) {  // whole warp
+  asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+// D (+)= A * B^T over the pair: M = 256 (each block holds 128 rows of A in its shared memory and the matching 128
+// lanes of D in its tensor memory), N columns of which each block's shared memory holds one half of B (the even
+// block the first half).  Issued by one thread of the even block; the descriptors are offsets into either block's
+// shared memory, so both blocks lay their operands out alike.
+__device__ __forceinline__ void umma_f16_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                              uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+      "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// One arrival on the mbarrier at this shared-memory offset in every block of `cta_mask` (bit = rank in the cluster)
+// once all tcgen05 operations issued so far by this thread are done.
+__device__ __forceinline__ void umma_commit_pair(uint64_t* bar, uint16_t cta_mask) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(
+                   smem_u32(bar)),
+               "h"(cta_mask)
+               : "memory");
+}
+// 2-D tiled load into this block's shared memory whose completion is counted on an mbarrier that may live in the
+// other block of the pair (`bar_cluster` is a shared::cluster address, see mapa_shared).
+__device__ __forceinline__ void tma_load_2d_pair(void* smem_dst, const CUtensorMap* map, int x, int y, uint32_t bar_cluster) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(
+          smem_u32(smem_dst)),
+      "l"(map), "r"(x), "r"(y), "r"(bar_cluster)
+      : "memory");
+}
+
+// One step of a copy-issuing thread as a single instruction sequence: test the NEXT stage's "free" barrier (result
+// wanted one step later), announce `expect_bytes` on `expect_bar` (skipped when 0), issue the 2-D tiled load, and only
+// then read the test's result - the test's latency would otherwise stall the in-order thread at every stage.
+// `bar_cluster` is the shared::cluster address of the barrier that counts the copy's bytes (it may live in the other
+// block of a pair: the cta_group::2 form).  Returns whether the next stage is already free.
+__device__ __forceinline__ bool tma_load_2d_pair_step(void* smem_dst, const CUtensorMap* map, int x, int y, uint32_t bar_cluster,
+                                                      uint64_t* expect_bar, uint32_t expect_bytes, uint64_t* next_free,
+                                                      uint32_t parity) {
+  uint32_t ready;
+  asm volatile(
+      "{\n\t.reg .pred r, e;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 r, [%8], %9;\n\t"
+      "setp.ne.b32 e, %7, 0;\n\t"
+      "@e mbarrier.arrive.expect_tx.shared::cta.b64 _, [%6], %7;\n\t"
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%1], [%2, {%3, %4}], [%5];\n\t"
+      "selp.u32 %0, 1, 0, r;\n\t}"
+      : "=r"(ready)
+      : "r"(smem_u32(smem_dst)), "l"(map), "r"(x), "r"(y), "r"(bar_cluster), "r"(smem_u32(expect_bar)), "r"(expect_bytes),
+        "r"(smem_u32(next_free)), "r"(parity)
+      : "memory");
+  return ready != 0;
+}
+
 // ---- thread-block clusters and distributed shared memory --------------------------------------
 __device__ __forceinline__ uint32_t cluster_ctarank() {
   uint32_t r;

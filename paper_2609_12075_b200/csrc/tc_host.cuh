@@ -4,6 +4,7 @@
 #include <cuda_runtime.h>
 
 #include "gemm_tc.cuh"
+#include "gemm_pair.cuh"
 
 namespace adit {
 namespace tc {
@@ -61,6 +62,7 @@ struct GemmPlan {
   uint32_t tmem_cols, ring_bytes;
   size_t smem_bytes;
   double est_us;  // the planner's estimate of the kernel's duration
+  bool pair = false;  // the two-SM kernel (gemm_pair_kernel): tile_tok tokens x 256 features per pair of blocks
 };
 
 // Tile shape and k-split (= cluster size) depend on the problem size and the device's SM count only,
@@ -159,6 +161,71 @@ static GemmPlan plan_gemm(int n_tok, int n_feat, int K, bool dual, int sm_count,
   return p;
 }
 
+// Rows of the token operand's TMA box: a block of the two-SM kernel brings in half a tile.
+static int token_box_rows(const GemmPlan& p) { return p.pair ? p.tile_tok / 2 : p.tile_tok; }
+
+// Plan for the two-SM kernel: a pair of blocks owns tiles of 256 features x tile_tok tokens.  The tile width minimises
+// rounds x (k-blocks x time per k-block + epilogue), in cycles: a k-block's products take 2 cycles per token (twice for
+// a gate/up pair) at the tensor peak, shared memory (128 bytes per cycle) has to take in the stage and feed every
+// product its weight rows and this block's half of the tokens, and the issuing thread needs about 45 cycles per
+// product.  The model is coarse: it prefers the widest tiles, which is what measured best where this kernel is used.
+// As for plan_gemm, nothing here depends on the call's SM budget.
+static GemmPlan plan_gemm_pair(int n_tok, int n_feat, int K, bool dual, int sm_count) {
+  GemmPlan p{};
+  const int nv = dual ? 2 : 1;
+  p.pair = true;
+  p.n_ftiles = (n_feat + TILE_F - 1) / TILE_F;
+  p.kb_total = K / TILE_K;
+  p.splits = 1; p.issuers = 1;
+  const int n_fpairs = (p.n_ftiles + 1) / 2, n_pairs = sm_count / 2 > 0 ? sm_count / 2 : 1;
+  double best = 1e30;
+  for (int nt = 1; nt <= 128; ++nt) {
+    const int tile = (((n_tok + nt - 1) / nt) + 15) / 16 * 16;
+    if (tile > 256) continue;
+    if (nt > 1 && tile < 32) break;
+    const int64_t rounds = ((int64_t)n_fpairs * nt + n_pairs - 1) / n_pairs;
+    const int acc_bufs = 2 * nv * tile <= 512 ? 2 : 1;
+    const double stage = nv * 16384.0 + tile * 64.0;
+    double t_kb = 2.0 * nv * tile;                                          // products
+    const double smem = (stage + nv * (16384.0 + tile * 64.0)) / 128.0;     // stage in + operand reads
+    if (smem > t_kb) t_kb = smem;
+    if (t_kb < 4.0 * nv * 45.0) t_kb = 4.0 * nv * 45.0;                     // issue rate of one thread
+    const double t_epi = 12.0 * tile * (dual ? 1.3 : 1.0);                  // about 0.2 us per 32 tokens
+    // with two accumulator buffers only the last tile's epilogue is exposed
+    const double t = acc_bufs == 2 ? rounds * p.kb_total * t_kb + t_epi : rounds * (p.kb_total * t_kb + t_epi);
+    if (t < best - 1e-9) { best = t; p.n_ttiles = nt; p.tile_tok = tile; p.acc_bufs = acc_bufs; }
+  }
+  p.est_us = 2.0 + best / 1900.0;  // (launch, set-up of the pair, first operands)
+  const size_t stage_bytes = (size_t)nv * TILE_F * TILE_K * 2 + (size_t)(p.tile_tok / 2) * TILE_K * 2;
+  p.stages = (int)(SMEM_BUDGET / stage_bytes);
+  if (p.stages > MAX_STAGES) p.stages = MAX_STAGES;
+  if ((int64_t)n_fpairs * p.n_ttiles <= n_pairs) {
+    // one tile per pair: a ring as deep as the tile's k-blocks is enough (the smaller footprint lets the next
+    // kernel's blocks become resident beside this one)
+    int kb_item = p.kb_total < 2 ? 2 : p.kb_total;
+    if (p.stages > kb_item) p.stages = kb_item;
+  }
+  p.ring_bytes = (uint32_t)(p.stages * stage_bytes);
+  p.smem_bytes = (size_t)p.ring_bytes + 1024;
+  uint32_t need = (uint32_t)(p.acc_bufs * nv * p.tile_tok), cols = 32;
+  while (cols < need) cols <<= 1;
+  p.tmem_cols = cols;
+  return p;
+}
+
+// The plan a projection runs with.  Measured on B200 at 816 and 1632 tokens, the two-SM kernel beats the one-SM kernel
+// (which has two issuing threads and finer tiles) only for the gate/up pair at the larger size - 33 against 36 us - and
+// for large plain products (8192 x 2048 x 2048: 54 against 62 us); the other projections of these sizes are bound by
+// fixed costs (set-up, first operands, the exposed epilogue of a single tile per block), where the pair's longer set-up
+// loses.  So: gate/up pairs from PAIR_DUAL_MIN_TOKENS tokens on go to the two-SM kernel, everything else to the
+// one-SM kernel with its k-split.  A function of the problem size and the device only.
+constexpr int PAIR_DUAL_MIN_TOKENS = 1024;
+static GemmPlan plan_projection(int n_tok, int n_feat, int K, bool dual, int sm_count, bool allow_pair) {
+  if (allow_pair && dual && n_tok >= PAIR_DUAL_MIN_TOKENS && sm_count >= 2 && (K / TILE_K) >= 2)
+    return plan_gemm_pair(n_tok, n_feat, K, dual, sm_count);
+  return plan_gemm(n_tok, n_feat, K, dual, sm_count, true);
+}
+
 // One instantiation per (gate/up pair, epilogue) x chunk width x k-split x issuing threads x instrumentation: a
 // launch then runs through (and has to fetch) only the code it needs.
 template <bool D, int E, typename F>
@@ -170,6 +237,28 @@ static cudaError_t for_gemm_variant(int idx, F&& f) {
     ADIT_V(8, 16, false, 1, true) ADIT_V(9, 32, false, 1, true) ADIT_V(10, 16, true, 1, true) ADIT_V(11, 32, true, 1, true)
     ADIT_V(12, 16, false, 2, true) ADIT_V(13, 32, false, 2, true) ADIT_V(14, 16, true, 2, true) ADIT_V(15, 32, true, 2, true)
 #undef ADIT_V
+    default: return cudaErrorInvalidValue;
+  }
+}
+template <bool D, int E, typename F>
+static cudaError_t for_pair_variant(int idx, F&& f) {
+  switch (idx) {
+    case 0: return f(gemm_pair_kernel<D, E, 16, false>);
+    case 1: return f(gemm_pair_kernel<D, E, 32, false>);
+    case 2: return f(gemm_pair_kernel<D, E, 16, true>);
+    case 3: return f(gemm_pair_kernel<D, E, 32, true>);
+    default: return cudaErrorInvalidValue;
+  }
+}
+template <typename F>
+static cudaError_t for_pair_kernel(bool dual, int epi, int idx, F&& f) {
+  if (dual) return for_pair_variant<true, EPI_GEGLU>(idx, f);
+  switch (epi) {
+    case EPI_STORE: return for_pair_variant<false, EPI_STORE>(idx, f);
+    case EPI_SILU_VEC: return for_pair_variant<false, EPI_SILU_VEC>(idx, f);
+    case EPI_STORE_F32: return for_pair_variant<false, EPI_STORE_F32>(idx, f);
+    case EPI_RESID_NORM: return for_pair_variant<false, EPI_RESID_NORM>(idx, f);
+    case EPI_EMBED_NORM: return for_pair_variant<false, EPI_EMBED_NORM>(idx, f);
     default: return cudaErrorInvalidValue;
   }
 }
@@ -203,11 +292,25 @@ static cudaError_t ensure_smem_attr() {
       });
       if (e != cudaSuccess) return e;
     }
+  for (int e6 = 0; e6 < 6; ++e6)
+    for (int idx = 0; idx < 4; ++idx) {
+      cudaError_t e = for_pair_kernel(e6 == 5, epis[e6], idx, [](auto kern) {
+        return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BUDGET + 1024);
+      });
+      if (e != cudaSuccess) return e;
+    }
   done = true;
   return cudaSuccess;
 }
 
 static int gemm_grid(const GemmPlan& p, int budget) {
+  if (p.pair) {  // pairs of blocks; a pair needs two SMs, so a budget of one is served with two
+    const int items = ((p.n_ftiles + 1) / 2) * p.n_ttiles;
+    int pairs = budget / 2;
+    if (pairs < 1) pairs = 1;
+    if (pairs > items) pairs = items;
+    return 2 * pairs;
+  }
   const int items = p.n_ftiles * p.n_ttiles;
   int clusters = budget / p.splits;
   if (clusters < 1) clusters = 1;
@@ -233,9 +336,9 @@ static cudaError_t launch_gemm(const CUtensorMap& map_w, const CUtensorMap& map_
     attr[na].val.programmaticStreamSerializationAllowed = 1;
     ++na;
   }
-  if (p.splits > 1) {
+  if (p.splits > 1 || p.pair) {
     attr[na].id = cudaLaunchAttributeClusterDimension;
-    attr[na].val.clusterDim.x = (unsigned)p.splits;
+    attr[na].val.clusterDim.x = p.pair ? 2u : (unsigned)p.splits;
     attr[na].val.clusterDim.y = 1;
     attr[na].val.clusterDim.z = 1;
     ++na;
@@ -244,6 +347,9 @@ static cudaError_t launch_gemm(const CUtensorMap& map_w, const CUtensorMap& map_
   cfg.numAttrs = na;
   // tokens per epilogue chunk: 32 for wide tiles that are a multiple of 32, else 16
   const bool wide = (p.tile_tok & 31) == 0 && p.tile_tok >= 96;
+  if (p.pair)
+    return for_pair_kernel(dual, g.epi, (wide ? 1 : 0) | ((g.dbg || g.trace) ? 2 : 0),
+                           [&](auto kern) { return cudaLaunchKernelEx(&cfg, kern, map_w, map_a, g); });
   const int idx = (wide ? 1 : 0) | (p.splits > 1 ? 2 : 0) | (p.issuers == 2 ? 4 : 0) | ((g.dbg || g.trace) ? 8 : 0);
   return for_gemm_kernel(dual, g.epi, idx, [&](auto kern) { return cudaLaunchKernelEx(&cfg, kern, map_w, map_a, g); });
 }

@@ -10,6 +10,10 @@ SHAPES = [
     (17, 128, 64, 0), (34, 384, 256, 0), (34, 384, 256, 3),
     (816, 2560, 1024, 0), (816, 1024, 2048, 0), (1632, 1024, 4096, 0), (408, 4608, 1536, 0),
     (50, 1000, 1024, 0), (300, 130, 192, 2),
+    # splits = -2: the two-SM kernel (pairs of thread blocks; 256 features x tile tokens per pair): one and several
+    # tiles per pair, an odd number of feature tiles, ragged token tails, rings shorter and longer than the k loop
+    (64, 256, 128, -2), (1632, 2560, 1024, -2), (1632, 1024, 4096, -2), (816, 1024, 2048, -2), (300, 130, 192, -2),
+    (500, 384, 256, -2), (408, 4608, 1536, -2), (8192, 2048, 2048, -2),
 ]
 
 
@@ -37,6 +41,21 @@ def test_projection_kernel_matches_fp32_matmul(adit, n_tok, n_feat, k, splits, b
     scale = ref.abs().max().item()
     assert torch.isfinite(out).all()
     assert err <= 2e-5 * k ** 0.5 * max(scale, 1.0) / 10 + 1e-4, (rc, err, scale)
+
+
+def test_two_sm_kernel_budget_does_not_change_a_single_bit(adit):
+    import torch
+    g = torch.Generator().manual_seed(2)
+    a = torch.randn(1632, 1024, generator=g).to(torch.bfloat16).cuda()
+    w = torch.randn(2560, 1024, generator=g).to(torch.bfloat16).cuda()
+    outs = []
+    for budget in (0, 1, 2, 7, 74, 148):  # (a pair needs two SMs: a budget of one is served with two)
+        out = torch.empty(1632, 2560, device="cuda")
+        rc = adit.lib.adit_debug_gemm(0, 1632, 2560, 1024, a.data_ptr(), w.data_ptr(), out.data_ptr(), -2, budget, None)
+        assert rc // 1000000 == 9, rc
+        outs.append(out.cpu().numpy())
+    for o in outs[1:]:
+        assert np.array_equal(o.view(np.uint32), outs[0].view(np.uint32))
 
 
 def test_budget_does_not_change_a_single_bit(adit):

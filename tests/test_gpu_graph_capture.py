@@ -1,5 +1,7 @@
 """adit_denoise recorded into the caller's CUDA graph (paper section 4.1.1: one graph per stage and batch size):
 replays must give the bits of direct calls on whatever the captured buffers hold at replay time."""
+import gc
+
 import numpy as np
 import pytest
 
@@ -30,7 +32,12 @@ def test_call_can_be_captured_and_replayed(persistent):
         s.synchronize()
     fresh = adit.ADiT(cfg, max_batch=len(plens), max_prefix_len=cap, flags=adit.FLAG_PERSISTENT_LOOP if persistent else 0)
     fresh.load_weights(W.make_weights(cfg, wl.seed))
-    with torch.cuda.graph(torch.cuda.CUDAGraph(), stream=s, capture_error_mode="thread_local"):
+    # (objects of earlier tests that are collected while a capture is open would free device memory inside it and
+    # invalidate the capture: collect them now)
+    gc.collect()
+    torch.cuda.synchronize()
+    refused = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(refused, stream=s, capture_error_mode="thread_local"):
         with pytest.raises(adit.AditError) as e:
             fresh.denoise(kv, wl.prefix_len, state, noise, steps, stream=s, out=out)
         assert e.value.code == adit.E_UNSUPPORTED
@@ -38,6 +45,7 @@ def test_call_can_be_captured_and_replayed(persistent):
     # warm-up outside the capture, then record
     direct0 = eng.denoise(kv, wl.prefix_len, state, noise, steps, stream=s, out=torch.empty_like(noise))
     s.synchronize()
+    gc.collect()
     with torch.cuda.graph(g, stream=s, capture_error_mode="thread_local"):
         eng.denoise(kv, wl.prefix_len, state, noise, steps, stream=s, out=out)
     g.replay()
@@ -56,3 +64,5 @@ def test_call_can_be_captured_and_replayed(persistent):
     assert torch.equal(out, direct1) and not torch.equal(direct1, direct0)
     assert eng.poll_status() == 0
     eng.close()
+    del g, refused
+    gc.collect()

@@ -327,6 +327,17 @@ def test_c4_full_size_budgets_and_sampled_requests(adit):
     assert np.isfinite(full).all()
     capped = gpu_run(adit, wl, w, eng=eng, kv=kv, sm_budget=64)
     assert np.array_equal(full.view(np.uint32), capped.view(np.uint32))
+    capped = gpu_run(adit, wl, w, eng=eng, kv=kv, sm_budget=1)   # (the two-SM gate/up kernel then runs as one pair)
+    assert np.array_equal(full.view(np.uint32), capped.view(np.uint32))
     eng.close()
     sample = [5, 31]
-    print("C4", check(full[sample], oracle(wl, w, subset=sample), "bf16", "C4"))
+    ref = oracle(wl, w, subset=sample)
+    print("C4", check(full[sample], ref, "bf16", "C4"))
+    # the same call with every projection on the one-SM kernel (at this size the gate/up pair otherwise runs on the
+    # two-SM kernel): another summation order, the same tolerance against the oracle
+    eng = adit.ADiT(wl.cfg, max_batch=wl.batch, max_prefix_len=wl.max_prefix_len, flags=adit.FLAG_ONE_SM_GEMM)
+    eng.load_weights(w)
+    one = gpu_run(adit, wl, w, eng=eng, kv=kv)
+    eng.close()
+    print("C4 one-SM projections", check(one[sample], ref, "bf16", "C4 one-SM"))
+    assert np.abs(one - full).max() <= 2e-2
