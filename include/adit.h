@@ -164,6 +164,37 @@ int adit_denoise_host(adit_handle* h, int B, const void* const* prefix_kv, const
                       const float* state_host, const float* noise_host, int K, int sm_budget,
                       void* stream, float* out_actions_host);
 
+/*
+ * Hidden-state hand-over (section 2.1: the VLM creates "hidden states or a small KV cache" for the
+ * ADiT).  Where the VLM hands over hidden states, the expert projects them to the per-layer prefix
+ * keys and values itself, once per call (they do not depend on the diffusion step), and the loop then
+ * runs on that cache as usual:
+ *   K_l = H Wk_l,  V_l = H Wv_l   for every layer l, H = hidden[b] [prefix_len[b], Dh]
+ * (no normalisation, bias or rotation here: H is used as handed over).
+ *
+ * adit_load_prefix_projection: the 2 * n_layers matrices, all in one call, named
+ *   layers.<l>.prefix_wk [Dh, KV]   layers.<l>.prefix_wv [Dh, KV]
+ * with one hidden width Dh (a multiple of 64) and KV = n_kv_heads * head_dim, columns head-major as for
+ * wk / wv.  Independent of adit_load_weights; a second call replaces the matrices.  Synchronises the
+ * device.  Errors: INVALID (NULL, a name missing or repeated, shapes), UNSUPPORTED (fp32 handles,
+ * ADIT_FLAG_REFERENCE_KERNELS, or together with ADIT_FLAG_SUFFIX_ROPE), CUDA.
+ *
+ * adit_project_prefix: enqueue the projection for B requests on `stream`.
+ *   hidden         HOST array of B DEVICE pointers, hidden[b] = [prefix_len[b], Dh] bf16, row-major,
+ *                  16-byte aligned (may be NULL where prefix_len[b] == 0)
+ *   prefix_len     HOST array of B lengths, 0 <= prefix_len[b] <= max_prefix_len
+ *   prefix_kv_out  HOST array of B DEVICE pointers to caches in adit_denoise's layout
+ *                  [n_layers][2][n_kv_heads][max_prefix_len][head_dim] bf16; rows < prefix_len[b] are
+ *                  written, rows beyond are left as they are (adit_denoise never reads them)
+ *   sm_budget      as in adit_denoise
+ * One tensor-core product per request (fp32 accumulation, results rounded to bf16); a request's
+ * cache depends on its own hidden states and length only.  Asynchronous; both host arrays are consumed
+ * before it returns.  Errors: INVALID, CAPACITY (B > max_batch), NOT_LOADED (no projection loaded), CUDA.
+ */
+int adit_load_prefix_projection(adit_handle* h, const adit_tensor* tensors, int n_tensors);
+int adit_project_prefix(adit_handle* h, int B, const void* const* hidden, const int32_t* prefix_len,
+                        void* const* prefix_kv_out, int sm_budget, void* stream);
+
 /* adit_destroy: synchronise the device and free everything the handle owns.  NULL is accepted. */
 int adit_destroy(adit_handle* h);
 

@@ -30,6 +30,10 @@ the following reading, taken step by step, one request at a time:
   suffix queries and keys of every head are rotated by the angles pos * 10000**(-2j/head_dim), j < head_dim/2,
   pairing channel j with channel j + head_dim/2, at position pos = prefix_len + (index of the token in the
   suffix); prefix keys are used as given (their producer has rotated them);
+* hidden-state hand-over (section 2.1 names hidden states beside the KV cache as what the VLM may hand over):
+  `project_prefix_kv` - the expert projects the handed-over hidden states H [P, Dh] to each layer's prefix keys
+  and values itself, K_l = H Wk_l, V_l = H Wv_l (no norm, bias or rotation), once per call; the loop then runs on
+  that cache;
 * GeGLU: tanh-approximate GELU on the gate times the up projection;
 * read-out: final RMSNorm, then Wout, bout, on the action tokens only.
 
@@ -44,7 +48,9 @@ permutation, padding and capacity invariance; time-embedding special values;
 for the variants: the masked attention against torch's masked attention and a
 scalar loop, the state token's independence of the action tokens; the rotary
 embedding against its closed form in two dimensions, norm preservation, the
-identity at position 0 and the dependence of a score on the position difference only.
+identity at position 0 and the dependence of a score on the position difference only;
+the hand-over projection against scalar loops and, with selection matrices as weights, against slices of the
+hidden states themselves.
 Parity unpinned: the behaviour of a *trained* model (no weights or reference
 outputs exist); the oracle pins the computation, not robot behaviour.
 """
@@ -127,6 +133,22 @@ def attention(q: np.ndarray, k_suffix: np.ndarray, v_suffix: np.ndarray,
             s[0, prefix_len + 1:] = -np.inf
         out[:, h, :] = softmax_rows(s) @ v_all
     return out
+
+
+def project_prefix_kv(cfg, hidden: np.ndarray, prefix_w: Dict[str, np.ndarray], max_prefix_len: int,
+                      pad_value: float = float("nan")) -> np.ndarray:
+    """Hidden-state hand-over (section 2.1): hidden [P, Dh] -> the request's prefix cache
+    [n_layers, 2, n_kv_heads, max_prefix_len, head_dim] with K_l = H Wk_l and V_l = H Wv_l in rows < P
+    (columns of the products are head-major: column = kv head * head_dim + channel); rows >= P hold pad_value."""
+    hidden = np.asarray(hidden, dtype=F64)
+    P = hidden.shape[0]
+    kv = np.full((cfg.n_layers, 2, cfg.n_kv_heads, max_prefix_len, cfg.head_dim), pad_value, dtype=F64)
+    for l in range(cfg.n_layers):
+        for which, leaf in enumerate(("prefix_wk", "prefix_wv")):
+            y = hidden @ np.asarray(prefix_w[f"layers.{l}.{leaf}"], dtype=F64)  # [P, n_kv_heads * head_dim]
+            for g in range(cfg.n_kv_heads):
+                kv[l, which, g, :P, :] = y[:, g * cfg.head_dim:(g + 1) * cfg.head_dim]
+    return kv
 
 
 def embed_tokens(cfg, w: Dict[str, np.ndarray], x: np.ndarray, state: np.ndarray, t: float) -> np.ndarray:

@@ -28,7 +28,7 @@ MAX_BATCH, MAX_STEPS = 64, 64
 EXPORTS = ["adit_create", "adit_load_weights", "adit_denoise", "adit_denoise_host", "adit_destroy",
            "adit_poll_status", "adit_last_cuda_error", "adit_kernel_launches", "adit_strerror",
            "adit_debug_copy", "adit_debug_gemm", "adit_debug_plan", "adit_debug_gemm_stamps", "adit_debug_attention", "adit_attention_static", "adit_profile_enable", "adit_profile_read", "adit_profile_class_name", "adit_trace_enable", "adit_trace_read",
-           "adit_bg_gemm_create", "adit_bg_gemm_create_kind", "adit_bg_gemm_launch", "adit_bg_gemm_destroy",
+           "adit_load_prefix_projection", "adit_project_prefix", "adit_bg_gemm_create", "adit_bg_gemm_create_kind", "adit_bg_gemm_launch", "adit_bg_gemm_destroy",
            "adit_debug_stream_read", "adit_attention_static_status", "adit_debug_stamps_selected",
            "adit_clear_status", "adit_uses_persistent_loop", "adit_debug_wait_limit", "adit_loop_trace_read"]
 
@@ -51,6 +51,8 @@ _DENOISE_ARGS = [C.c_void_p, C.c_int, C.POINTER(C.c_void_p), C.POINTER(C.c_int32
                  C.c_int, C.c_int, C.c_void_p, C.c_void_p]
 lib.adit_denoise.argtypes = _DENOISE_ARGS
 lib.adit_denoise_host.argtypes = _DENOISE_ARGS
+lib.adit_load_prefix_projection.argtypes = [C.c_void_p, C.POINTER(Tensor), C.c_int]
+lib.adit_project_prefix.argtypes = [C.c_void_p, C.c_int, C.POINTER(C.c_void_p), C.POINTER(C.c_int32), C.POINTER(C.c_void_p), C.c_int, C.c_void_p]
 lib.adit_destroy.argtypes = [C.c_void_p]
 lib.adit_poll_status.argtypes = [C.c_void_p]
 lib.adit_last_cuda_error.argtypes = [C.c_void_p]
@@ -148,6 +150,30 @@ class ADiT:
             arr[i] = Tensor(name=name.encode(), data=w.ctypes.data, dtype=DTYPE_FP32, ndim=w.ndim, shape=shape,
                             on_device=0)
         self._check(lib.adit_load_weights(self._h, arr, len(weights)))
+
+    # -- hidden-state hand-over ---------------------------------------------------------------
+    def load_prefix_projection(self, weights: Dict[str, np.ndarray]):
+        """weights: layers.<l>.prefix_wk / prefix_wv -> float32 [Dh, KV] (all layers, one call)."""
+        keep, arr = [], (Tensor * len(weights))()
+        for i, (name, w) in enumerate(weights.items()):
+            w = np.ascontiguousarray(w, dtype=np.float32)
+            keep.append(w)
+            shape = (C.c_int64 * 4)(*(list(w.shape) + [1] * (4 - w.ndim)))
+            arr[i] = Tensor(name=name.encode(), data=w.ctypes.data, dtype=DTYPE_FP32, ndim=w.ndim, shape=shape,
+                            on_device=0)
+        self._check(lib.adit_load_prefix_projection(self._h, arr, len(weights)))
+
+    def project_prefix(self, hidden: Sequence, prefix_len: Sequence[int], prefix_kv_out: Sequence, sm_budget: int = 0,
+                       stream=None):
+        """hidden[b]: bf16 cuda [prefix_len[b], Dh]; writes rows < prefix_len[b] of the caches prefix_kv_out[b] (async)."""
+        import torch
+        n = len(prefix_len)
+        hp = (C.c_void_p * n)(*[int(t.data_ptr()) if t is not None else None for t in hidden])
+        op = (C.c_void_p * n)(*[int(t.data_ptr()) for t in prefix_kv_out])
+        lens = (C.c_int32 * n)(*[int(v) for v in prefix_len])
+        st = stream if stream is not None else torch.cuda.current_stream(self.device)
+        self._check(lib.adit_project_prefix(self._h, n, hp, lens, op, int(sm_budget), C.c_void_p(st.cuda_stream)))
+        return prefix_kv_out
 
     # -- the call -----------------------------------------------------------------------------
     @staticmethod

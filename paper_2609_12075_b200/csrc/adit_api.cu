@@ -80,6 +80,10 @@ struct adit_handle {
   int* status_host = 0;  // pinned, device-visible status word
   int* status_dev = 0;   // its device address
   float2* rope_tab = 0;  // cos/sin per suffix token row and channel pair (variant ADIT_FLAG_SUFFIX_ROPE)
+  // hidden-state hand-over (adit_project_prefix): the prefix K/V projections of every layer as one matrix
+  void* Wp = 0;                // bf16 [n_layers * 2 * KV, prefix_hidden_dim], rows ordered (layer, K then V, kv head, channel)
+  int prefix_hidden_dim = 0;   // 0 until adit_load_prefix_projection has run
+  CUtensorMap m_wp;
   int64_t launches = 0;
   int last_cuda = 0;
   bool profiling = false;
@@ -477,6 +481,122 @@ extern "C" int adit_load_weights(adit_handle* h, const adit_tensor* tensors, int
   }
   if (h->raw.size() == n_expected_tensors(h->cfg))
     return h->cfg.dtype == ADIT_DTYPE_BF16 ? pack_all<bf16>(h) : pack_all<float>(h);
+  return ADIT_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Hidden-state hand-over: the expert projects the prefix K/V itself, once per call
+// ---------------------------------------------------------------------------------------------
+// Copies one tensor to a fresh device buffer as fp32 (the caller frees it).
+static int stage_f32(adit_handle* h, const adit_tensor& t, int64_t n, float** out) {
+  float* dst = nullptr;
+  CU_TRY(h, cudaMalloc((void**)&dst, (size_t)n * 4));
+  const cudaMemcpyKind kind = t.on_device ? cudaMemcpyDeviceToDevice : cudaMemcpyHostToDevice;
+  cudaError_t e;
+  if (t.dtype == ADIT_DTYPE_FP32) {
+    e = cudaMemcpy(dst, t.data, (size_t)n * 4, kind);
+  } else {
+    uint16_t* tmp = nullptr;
+    e = cudaMalloc((void**)&tmp, (size_t)n * 2);
+    if (e == cudaSuccess) e = cudaMemcpy(tmp, t.data, (size_t)n * 2, kind);
+    if (e == cudaSuccess) {
+      bf16_bits_to_f32_kernel<<<(unsigned)((n + 255) / 256), 256>>>(tmp, dst, n);
+      e = cudaDeviceSynchronize();
+    }
+    if (tmp) cudaFree(tmp);
+  }
+  if (e != cudaSuccess) { cudaFree(dst); h->last_cuda = (int)e; return ADIT_E_CUDA; }
+  *out = dst;
+  return ADIT_OK;
+}
+
+extern "C" int adit_load_prefix_projection(adit_handle* h, const adit_tensor* tensors, int n_tensors) {
+  if (!h || !tensors) return ADIT_E_INVALID;
+  const adit_config& c = h->cfg;
+  if (use_reference_kernels(c)) return ADIT_E_UNSUPPORTED;  // (tensor-core path only)
+  if (c.flags & ADIT_FLAG_SUFFIX_ROPE) return ADIT_E_UNSUPPORTED;  // (prefix keys would need their own rotation)
+  const int L = c.n_layers, KV = c.n_kv_heads * c.head_dim;
+  if (n_tensors != 2 * L) return ADIT_E_INVALID;
+  // every layer's prefix_wk and prefix_wv exactly once, all [Dh, KV] with one Dh that is a multiple of 64
+  std::vector<int> slot(2 * L, -1);
+  int64_t Dh = 0;
+  for (int i = 0; i < n_tensors; ++i) {
+    const adit_tensor& t = tensors[i];
+    if (!t.name || !t.data || t.ndim != 2 || t.shape[1] != KV) return ADIT_E_INVALID;
+    if (t.dtype != ADIT_DTYPE_FP32 && t.dtype != ADIT_DTYPE_BF16) return ADIT_E_INVALID;
+    const std::string name = t.name;
+    if (name.rfind("layers.", 0) != 0) return ADIT_E_INVALID;
+    const size_t dot = name.find('.', 7);
+    if (dot == std::string::npos || dot == 7) return ADIT_E_INVALID;
+    for (size_t k = 7; k < dot; ++k)
+      if (name[k] < '0' || name[k] > '9') return ADIT_E_INVALID;
+    const long l = strtol(name.substr(7, dot - 7).c_str(), nullptr, 10);
+    const std::string leaf = name.substr(dot + 1);
+    if (l < 0 || l >= L || (leaf != "prefix_wk" && leaf != "prefix_wv")) return ADIT_E_INVALID;
+    const int s = (int)l * 2 + (leaf == "prefix_wv" ? 1 : 0);
+    if (slot[s] >= 0) return ADIT_E_INVALID;
+    slot[s] = i;
+    if (Dh == 0) Dh = t.shape[0];
+    if (t.shape[0] != Dh) return ADIT_E_INVALID;
+  }
+  if (Dh < 64 || (Dh % 64) || Dh > (1 << 20)) return ADIT_E_INVALID;
+  CU_TRY(h, cudaSetDevice(h->device));
+  CU_TRY(h, cudaDeviceSynchronize());  // (a call still using the previous matrix has finished)
+  void* wp = nullptr;
+  CU_TRY(h, cudaMalloc(&wp, (size_t)2 * L * KV * Dh * 2));
+  for (int s = 0; s < 2 * L; ++s) {
+    float* src = nullptr;
+    int rc = stage_f32(h, tensors[slot[s]], Dh * KV, &src);
+    if (rc) { cudaFree(wp); return rc; }
+    const int64_t n = Dh * KV;
+    // [in = Dh, out = KV] -> rows s * KV .. of the [out, in] matrix
+    pack_rows_kernel<bf16><<<(unsigned)((n + 255) / 256), 256>>>(src, (int)Dh, KV, nullptr, (bf16*)wp, (int64_t)s * KV, (int)Dh, 0, 0);
+    cudaError_t e = cudaDeviceSynchronize();
+    cudaFree(src);
+    if (e != cudaSuccess) { cudaFree(wp); h->last_cuda = (int)e; return ADIT_E_CUDA; }
+  }
+  if (!tc::make_map_bf16(&h->m_wp, wp, (uint64_t)2 * L * KV, (uint64_t)Dh, tc::TILE_F)) { cudaFree(wp); return ADIT_E_CUDA; }
+  if (h->Wp) {
+    for (auto& q : h->allocs)
+      if (q == h->Wp) { cudaFree(q); q = nullptr; }
+  }
+  h->allocs.push_back(wp);
+  h->Wp = wp;
+  h->prefix_hidden_dim = (int)Dh;
+  return ADIT_OK;
+}
+
+extern "C" int adit_project_prefix(adit_handle* h, int B, const void* const* hidden, const int32_t* prefix_len,
+                                   void* const* prefix_kv_out, int sm_budget, void* stream) {
+  if (!h || !hidden || !prefix_len || !prefix_kv_out || B < 1) return ADIT_E_INVALID;
+  const adit_config& c = h->cfg;
+  if (B > c.max_batch) return ADIT_E_CAPACITY;
+  if (!h->Wp) return ADIT_E_NOT_LOADED;
+  for (int b = 0; b < B; ++b) {
+    if (prefix_len[b] < 0 || prefix_len[b] > c.max_prefix_len) return ADIT_E_INVALID;
+    if (prefix_len[b] > 0 && (!hidden[b] || !prefix_kv_out[b])) return ADIT_E_INVALID;
+    if (((uintptr_t)hidden[b] & 15) || ((uintptr_t)prefix_kv_out[b] & 15)) return ADIT_E_INVALID;
+  }
+  CU_TRY(h, cudaSetDevice(h->device));
+  cudaStream_t st = (cudaStream_t)stream;
+  const int L = c.n_layers, KV = c.n_kv_heads * c.head_dim, Dh = h->prefix_hidden_dim, NF = 2 * L * KV;
+  const int G = (sm_budget <= 0 || sm_budget >= h->sm_count) ? h->sm_count : sm_budget;
+  for (int b = 0; b < B; ++b) {
+    const int P = prefix_len[b];
+    if (P == 0) continue;
+    // one product per request: [P, Dh] x [NF, Dh]^T, written straight into the cache's planes.  The plan depends on
+    // this request's length and the device only, so a request's cache never depends on its neighbours.
+    const tc::GemmPlan p = tc::plan_gemm(P, NF, Dh, false, h->sm_count, true);
+    CUtensorMap ma;
+    if (!tc::make_map_bf16(&ma, hidden[b], (uint64_t)P, (uint64_t)Dh, p.tile_tok)) return ADIT_E_CUDA;
+    tc::GemmArgs g{};
+    g.n_feat = NF; g.n_tok = P; g.epi = tc::EPI_STORE_PLANES; g.out = prefix_kv_out[b];
+    g.plane_w = c.head_dim; g.plane_stride = (int64_t)c.max_prefix_len * c.head_dim;
+    g.status = h->status_dev;
+    ProfScope ps(h, KC_PROLOGUE, st);
+    CU_TRY(h, tc::launch_gemm(h->m_wp, ma, p, false, g, G, st, false));
+    h->launches++;
+  }
   return ADIT_OK;
 }
 

@@ -40,7 +40,7 @@ constexpr int MAX_STAGES = 12;
 constexpr int GEMM_THREADS = 256;
 constexpr int SMEM_BUDGET = 216 * 1024;  // dynamic shared memory: stage ring + cluster exchange buffer
 
-enum : int { EPI_RESID_NORM = 6, EPI_EMBED_NORM = 7 };
+enum : int { EPI_RESID_NORM = 6, EPI_EMBED_NORM = 7, EPI_STORE_PLANES = 8 };
 
 struct GemmArgs {
   int n_feat;    // output features (DUAL: per matrix; the packed matrix has 2 * n_feat rows)
@@ -69,6 +69,8 @@ struct GemmArgs {
   int ssq_ld;
   float eps;
   int horizon;           // EPI_EMBED_NORM: action row m -> token row m + m / horizon + 1
+  int plane_w;           // EPI_STORE_PLANES: feature f of token t goes to out[(f / plane_w) * plane_stride + t * plane_w + f % plane_w]
+  int64_t plane_stride;  //   (bf16; a K/V cache laid out as planes of [rows][plane_w]); tokens >= n_tok are not stored
   int* status;           // device-visible status word (ADIT_E_TIMEOUT = -6 on an expired wait)
   unsigned long long* dbg;  // optional [grid][16] globaltimer stamps (test aid)
   unsigned long long* trace;  // optional [grid][4]: block start, predecessor-wait released, end, last accumulator complete (%globaltimer ns)
@@ -162,7 +164,13 @@ __device__ __forceinline__ void finalize_chunk(const GemmArgs& g, const float (&
   if constexpr (EPI != EPI_RESID_NORM && EPI != EPI_EMBED_NORM) {
     if (!f_ok) return;
     const int64_t ld = g.ldo;
-    if constexpr (EPI == EPI_STORE_F32) {
+    if constexpr (EPI == EPI_STORE_PLANES) {
+      // (the only epilogue whose destination has no padding rows: a token past the end would land in the next plane)
+      bf16* p = (bf16*)g.out + (int64_t)(f / g.plane_w) * g.plane_stride + (f % g.plane_w) + (int64_t)tok_base * g.plane_w;
+#pragma unroll
+      for (int j = 0; j < NT; ++j)
+        if (tok_base + j < g.n_tok) p[(int64_t)j * g.plane_w] = __float2bfloat16_rn(v[j]);
+    } else if constexpr (EPI == EPI_STORE_F32) {
       float* p = (float*)g.out + (int64_t)tok_base * ld + f;
       const float b = g.bias ? g.bias[f] : 0.f;
 #pragma unroll

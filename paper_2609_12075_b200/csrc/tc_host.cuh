@@ -271,6 +271,7 @@ static cudaError_t for_gemm_kernel(bool dual, int epi, int idx, F&& f) {
     case EPI_STORE_F32: return for_gemm_variant<false, EPI_STORE_F32>(idx, f);
     case EPI_RESID_NORM: return for_gemm_variant<false, EPI_RESID_NORM>(idx, f);
     case EPI_EMBED_NORM: return for_gemm_variant<false, EPI_EMBED_NORM>(idx, f);
+    case EPI_STORE_PLANES: return for_gemm_variant<false, EPI_STORE_PLANES>(idx, f);
     default: return cudaErrorInvalidValue;
   }
 }
@@ -284,8 +285,8 @@ static cudaError_t ensure_smem_attr() {
   bool unused = false;
   bool& done = (dev >= 0 && dev < 64) ? done_dev[dev] : unused;
   if (done) return cudaSuccess;
-  const int epis[6] = {EPI_STORE, EPI_SILU_VEC, EPI_STORE_F32, EPI_RESID_NORM, EPI_EMBED_NORM, EPI_GEGLU};
-  for (int e6 = 0; e6 < 6; ++e6)
+  const int epis[7] = {EPI_STORE, EPI_SILU_VEC, EPI_STORE_F32, EPI_RESID_NORM, EPI_EMBED_NORM, EPI_GEGLU, EPI_STORE_PLANES};
+  for (int e6 = 0; e6 < 7; ++e6)
     for (int idx = 0; idx < 16; ++idx) {
       cudaError_t e = for_gemm_kernel(e6 == 5, epis[e6], idx, [](auto kern) {
         return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BUDGET + 1024);

@@ -140,6 +140,26 @@ def make_weights(cfg: ADiTConfig, seed: int) -> Dict[str, np.ndarray]:
     return out
 
 
+def make_prefix_projection(cfg: ADiTConfig, seed: int, hidden_dim: int) -> Dict[str, np.ndarray]:
+    """Random-initialised prefix K/V projections of the hidden-state hand-over: layers.<l>.prefix_wk / prefix_wv
+    [hidden_dim, n_kv_heads * head_dim], float32 (bf16-representable), scaled so that the projected keys and values
+    have about unit variance like the generated caches."""
+    out: Dict[str, np.ndarray] = {}
+    kv = cfg.n_kv_heads * cfg.head_dim
+    for l in range(cfg.n_layers):
+        for j, leaf in enumerate(("prefix_wk", "prefix_wv")):
+            w = _rng(seed, 50000 + 2 * l + j).standard_normal((hidden_dim, kv)).astype(np.float32)
+            out[f"layers.{l}.{leaf}"] = round_to_bf16(w * np.float32(1.0 / np.sqrt(hidden_dim)))
+    return out
+
+
+def make_prefix_hidden(seed: int, b: int, prefix_len: int, hidden_dim: int) -> np.ndarray:
+    """Hidden states the VLM stand-in hands over for request ``b``: float32 [prefix_len, hidden_dim], unit variance,
+    bf16-representable; depends on (seed, b) only."""
+    g = _rng(seed, 70000 + b)
+    return round_to_bf16(g.standard_normal((prefix_len, hidden_dim)).astype(np.float32))
+
+
 @dataclass
 class Workload:
     """One batch of requests for ``adit_denoise``.

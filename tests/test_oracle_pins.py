@@ -485,6 +485,51 @@ def test_suffix_rope_changes_the_layer_and_reduces_to_plain_at_identity_position
 
 # ---- the full configurations run and are healthy --------------------------------------------
 
+def test_prefix_projection_against_scalar_loops_and_selection_weights():
+    """P14: the hidden-state hand-over.  (a) every cache element recomputed by a scalar triple loop that indexes the
+    cache layout itself; (b) with selection matrices as weights, keys are the first and values the last KV
+    columns of the hidden states, reversed for the values - a transposed operand, a swapped K/V plane or a
+    head-minor column order fails one of them; (c) rows at or beyond the prefix length keep the padding."""
+    cfg = SMALL
+    rng = np.random.default_rng(140)
+    Dh, P, cap = 12, 5, 7
+    KV = cfg.n_kv_heads * cfg.head_dim
+    H = rng.standard_normal((P, Dh))
+    pw = {f"layers.{l}.{leaf}": rng.standard_normal((Dh, KV)) for l in range(cfg.n_layers) for leaf in ("prefix_wk", "prefix_wv")}
+    kv = O.project_prefix_kv(cfg, H, pw, cap, pad_value=-7.0)
+    assert kv.shape == (cfg.n_layers, 2, cfg.n_kv_heads, cap, cfg.head_dim)
+    for l in range(cfg.n_layers):
+        for which, leaf in enumerate(("prefix_wk", "prefix_wv")):
+            Wm = pw[f"layers.{l}.{leaf}"]
+            for g in range(cfg.n_kv_heads):
+                for p in range(P):
+                    for c in range(cfg.head_dim):
+                        acc = 0.0
+                        for i in range(Dh):
+                            acc += H[p, i] * Wm[i, g * cfg.head_dim + c]
+                        assert abs(kv[l, which, g, p, c] - acc) < 1e-12
+    assert np.all(kv[:, :, :, P:, :] == -7.0)
+    # (b) selection weights
+    Dh2 = 2 * KV
+    H2 = rng.standard_normal((P, Dh2))
+    sel_k = np.zeros((Dh2, KV)); sel_v = np.zeros((Dh2, KV))
+    for j in range(KV):
+        sel_k[j, j] = 1.0                 # key column j = hidden column j
+        sel_v[Dh2 - 1 - j, j] = 1.0       # value column j = hidden column Dh2 - 1 - j
+    pw2 = {}
+    for l in range(cfg.n_layers):
+        pw2[f"layers.{l}.prefix_wk"] = sel_k * (l + 1)
+        pw2[f"layers.{l}.prefix_wv"] = sel_v * (l + 1)
+    kv2 = O.project_prefix_kv(cfg, H2, pw2, P)
+    for l in range(cfg.n_layers):
+        for g in range(cfg.n_kv_heads):
+            lo = g * cfg.head_dim
+            np.testing.assert_allclose(kv2[l, 0, g], (l + 1) * H2[:, lo:lo + cfg.head_dim], atol=0, rtol=0)
+            np.testing.assert_allclose(kv2[l, 1, g], (l + 1) * H2[:, ::-1][:, lo:lo + cfg.head_dim], atol=0, rtol=0)
+    # an empty prefix projects to nothing
+    assert np.all(np.isnan(O.project_prefix_kv(cfg, np.zeros((0, Dh)), pw, 3)))
+
+
 def test_config_c1_runs_and_signal_is_healthy():
     wl = W.config_c1()
     w = W.make_weights(wl.cfg, wl.seed)
