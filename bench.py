@@ -502,30 +502,48 @@ def run_budget_sweep(args):
         roof[str(budget)] = {"stream_read_gbs": read_gbs, "floor_ms_per_call": floor_ms,
                              "bound": "hbm" if work["step_bytes"] / (read_gbs * 1e9) >= work["step_flops"] / tc else "tensor"}
     for budget in [int(b) for b in args.budgets.split(",")]:
-        for load in (False, True):
+        # load: "" = none; "+load" = the stand-in's grid capped to the SMs outside the budget (persistent-grid form, the
+        # call's own grids capped to the budget); "+green" = the stand-in's full grid on a stream that the driver
+        # confines to the SMs outside the budget (green context, section 4.1.2), the call itself unrestricted
+        modes = ["", "+load"] + (["+green"] if args.green and budget < n_sm else [])
+        for mode in modes:
             lat = []
             load_sms = n_sm - budget if budget < n_sm else 0        # budget = all SMs: the load is not capped
             est_ms = None
+            green = None
+            if mode == "+green":
+                try:
+                    green = adit.GreenStream(load_sms)
+                except adit.AditError as e:
+                    results[f"{budget}+green"] = {"unavailable": str(e)}
+                    continue
+            ls = green.stream if green else s_load
             for i in range(args.warmup + args.steps):
-                if load:
+                if mode:
                     # keep the load stream busy well past the end of this call
                     per_iter = bg_ms_full * (n_sm / max(load_sms, 1) if load_sms else 2.0)
                     need_ms = (est_ms or 200.0) * 2.0
-                    bg.launch(max(4, int(need_ms / per_iter)), load_sms, s_load)
+                    bg.launch(max(4, int(need_ms / per_iter)), 0 if green else load_sms, ls)
                 a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                 a.record(s_adit)
-                eng.denoise(kv, base.prefix_len, st_in, nz, base.n_steps, sm_budget=budget, stream=s_adit, out=out)
+                eng.denoise(kv, base.prefix_len, st_in, nz, base.n_steps, sm_budget=0 if green else budget, stream=s_adit, out=out)
                 b.record(s_adit)
                 b.synchronize()
                 est_ms = a.elapsed_time(b)
                 if i >= args.warmup:
                     lat.append(est_ms)
             torch.cuda.synchronize()
+            if green:
+                load_granted = green.sm_count
+                green.close()
             lat = np.array(lat)
-            results[f"{budget}{'+load' if load else ''}"] = {
+            results[f"{budget}{mode}"] = {
                 "p50_ms": float(np.percentile(lat, 50)), "p99_ms": float(np.percentile(lat, 99)),
                 "chunks_per_s": base.batch / (float(lat.mean()) * 1e-3),
                 "roofline_frac_at_budget": roof[str(budget)]["floor_ms_per_call"] / float(np.percentile(lat, 50))}
+            if mode == "+green":  # (the call itself is not confined: no roofline of a budget applies)
+                results[f"{budget}{mode}"]["load_sms_granted"] = load_granted
+                results[f"{budget}{mode}"]["roofline_frac_at_budget"] = None
     assert eng.poll_status() == 0
     budgets = [int(b) for b in args.budgets.split(",")]
     ratios = {}
@@ -538,7 +556,8 @@ def run_budget_sweep(args):
                 ratios[f"halving_p99_{lo}_vs_{hi}_idle"] = results[f"{lo}"]["p99_ms"] / results[f"{hi}"]["p99_ms"]
     print(json.dumps({"metric": "adit_chunk_latency_vs_sm_budget", "unit": "ms", "config": {
         "workload": base.name, "batch": base.batch, "euler_steps": base.n_steps,
-        "load": "bf16 GEMM 8192x2048x2048 looping on a second stream, grid capped to the SMs outside the budget",
+        "load": "bf16 GEMM 8192x2048x2048 looping on a second stream, grid capped to the SMs outside the budget ('+load'); "
+                "with --green also its full grid on a green-context stream of those SMs while the call runs unrestricted ('+green')",
         "bg_gemm_ms_full_chip": bg_ms_full}, "steps": args.steps, "warmup": args.warmup, "n_sm": n_sm,
         "results": results, "ratios": ratios, "roofline_per_budget": roof}))
     bg.close()
@@ -694,6 +713,7 @@ def main():
     ap.add_argument("--no-trace", action="store_true", help="skip the in-situ timeline of one call")
     ap.add_argument("--no-extra", action="store_true", help="skip the brief runs of the other batch sizes (c3, c4)")
     ap.add_argument("--no-graph", action="store_true", help="enqueue kernels one by one (ADIT_FLAG_NO_GRAPH): for profilers")
+    ap.add_argument("--green", action="store_true", help="sweep: also run the load on a green-context stream confined to the SMs outside the budget, the call unrestricted")
     ap.add_argument("--one-sm-gemm", action="store_true", help="projections on the one-SM kernel at every batch size (ADIT_FLAG_ONE_SM_GEMM): comparison")
     ap.add_argument("--persistent", action="store_true", help="small batches as one persistent kernel (ADIT_FLAG_PERSISTENT_LOOP)")
     ap.add_argument("--latency-calls", type=int, default=None, help="calls sampled for p50/p99 (default 1000 at batch 1)")

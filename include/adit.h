@@ -377,6 +377,22 @@ int adit_debug_plan(int n_tok, int n_feat, int k, int dual, int sm_count, int32_
 int adit_debug_stream_read(int device, size_t bytes, int sm_count, int iters, double* gb_per_s);
 
 /*
+ * adit_green_stream_*: a stream whose kernels the driver confines to a partition of at least
+ * `sm_count` SMs (a green context; section 4.1.2 restricts the VLM stage's stream this way, in
+ * multiples of 8 SMs).  The alternative to the sm_budget argument, which caps the grids of this
+ * library's own persistent kernels: a green stream also confines kernels that were not written for a
+ * budget.  create returns UNSUPPORTED where the driver has no green contexts and CAPACITY when the
+ * device has fewer SMs; handle gives the cudaStream_t, sm_count the size of the partition the
+ * driver granted (rounded up to its granularity).  destroy synchronises the stream first.  Nothing
+ * outlives the process, and the rest of the device keeps running on all SMs.
+ */
+typedef struct adit_green_stream adit_green_stream;
+int adit_green_stream_create(int device, int sm_count, adit_green_stream** out);
+void* adit_green_stream_handle(adit_green_stream* g);
+int adit_green_stream_sm_count(adit_green_stream* g);
+int adit_green_stream_destroy(adit_green_stream* g);
+
+/*
  * adit_bg_gemm_*: a looping bf16 GEMM C[m,n] = A[m,k] B[n,k]^T on a capped number of SMs, the
  * stand-in for the VLM stage that shares the GPU with the ADiT stream (section 4.1.2: the VLM
  * stream is restricted to a number of SMs so that the ADiT kernels always find free ones).

@@ -28,7 +28,7 @@ MAX_BATCH, MAX_STEPS = 64, 64
 EXPORTS = ["adit_create", "adit_load_weights", "adit_denoise", "adit_denoise_host", "adit_destroy",
            "adit_poll_status", "adit_last_cuda_error", "adit_kernel_launches", "adit_strerror",
            "adit_debug_copy", "adit_debug_gemm", "adit_debug_plan", "adit_debug_gemm_stamps", "adit_debug_attention", "adit_attention_static", "adit_profile_enable", "adit_profile_read", "adit_profile_class_name", "adit_trace_enable", "adit_trace_read",
-           "adit_load_prefix_projection", "adit_project_prefix", "adit_bg_gemm_create", "adit_bg_gemm_create_kind", "adit_bg_gemm_launch", "adit_bg_gemm_destroy",
+           "adit_load_prefix_projection", "adit_project_prefix", "adit_green_stream_create", "adit_green_stream_handle", "adit_green_stream_sm_count", "adit_green_stream_destroy", "adit_bg_gemm_create", "adit_bg_gemm_create_kind", "adit_bg_gemm_launch", "adit_bg_gemm_destroy",
            "adit_debug_stream_read", "adit_attention_static_status", "adit_debug_stamps_selected",
            "adit_clear_status", "adit_uses_persistent_loop", "adit_debug_wait_limit", "adit_loop_trace_read"]
 
@@ -88,6 +88,11 @@ lib.adit_debug_wait_limit.argtypes = [C.c_void_p, C.c_int, C.c_int]
 lib.adit_loop_trace_read.argtypes = [C.c_void_p, C.POINTER(C.c_int64), C.c_int64]
 lib.adit_loop_trace_read.restype = C.c_int64
 lib.adit_bg_gemm_create.argtypes = [C.c_int, C.c_int, C.c_int, C.c_int, C.POINTER(C.c_void_p)]
+lib.adit_green_stream_create.argtypes = [C.c_int, C.c_int, C.POINTER(C.c_void_p)]
+lib.adit_green_stream_handle.argtypes = [C.c_void_p]
+lib.adit_green_stream_handle.restype = C.c_void_p
+lib.adit_green_stream_sm_count.argtypes = [C.c_void_p]
+lib.adit_green_stream_destroy.argtypes = [C.c_void_p]
 lib.adit_bg_gemm_create_kind.argtypes = [C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, C.POINTER(C.c_void_p)]
 lib.adit_bg_gemm_launch.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_void_p]
 lib.adit_bg_gemm_destroy.argtypes = [C.c_void_p]
@@ -294,6 +299,31 @@ def upload_prefix_kv(wl: W.Workload, device: int = 0) -> List:
     import torch
     dt = torch.bfloat16 if wl.cfg.dtype == "bf16" else torch.float32
     return [torch.from_numpy(kv).to(dt).to(f"cuda:{device}") for kv in wl.prefix_kv]
+
+
+class GreenStream:
+    """A stream confined by the driver to a partition of at least `sm_count` SMs (green context)."""
+
+    def __init__(self, sm_count: int, device: int = 0):
+        import torch
+        self._g = C.c_void_p()
+        rc = lib.adit_green_stream_create(device, int(sm_count), C.byref(self._g))
+        if rc != OK:
+            self._g = C.c_void_p()
+            raise AditError(rc)
+        self.sm_count = int(lib.adit_green_stream_sm_count(self._g))
+        self.stream = torch.cuda.ExternalStream(int(lib.adit_green_stream_handle(self._g)), device=device)
+
+    def close(self):
+        if self._g:
+            lib.adit_green_stream_destroy(self._g)
+            self._g = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
 
 
 class BackgroundGemm:

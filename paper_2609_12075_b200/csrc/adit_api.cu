@@ -1744,6 +1744,67 @@ extern "C" int adit_debug_stream_read(int device, size_t bytes, int sm_count, in
 }
 
 // ---------------------------------------------------------------------------------------------
+// A stream confined to an SM partition by the driver (green context): the paper's own way of restricting the VLM stage
+// ---------------------------------------------------------------------------------------------
+struct adit_green_stream {
+  int device;
+  CUgreenCtx ctx;
+  CUstream stream;
+  int sm_count;
+};
+
+template <typename F>
+static F driver_fn(const char* name) {
+  void* p = nullptr;
+  cudaDriverEntryPointQueryResult q;
+  if (cudaGetDriverEntryPoint(name, &p, cudaEnableDefault, &q) != cudaSuccess || q != cudaDriverEntryPointSuccess) return nullptr;
+  return (F)p;
+}
+
+extern "C" int adit_green_stream_create(int device, int sm_count, adit_green_stream** out) {
+  if (!out || sm_count < 1) return ADIT_E_INVALID;
+  if (cudaSetDevice(device) != cudaSuccess) return ADIT_E_CUDA;
+  if (cudaFree(0) != cudaSuccess) return ADIT_E_CUDA;  // (the primary context exists)
+  auto get_res = driver_fn<CUresult (*)(CUdevice, CUdevResource*, CUdevResourceType)>("cuDeviceGetDevResource");
+  auto split = driver_fn<CUresult (*)(CUdevResource*, unsigned int*, const CUdevResource*, CUdevResource*, unsigned int, unsigned int)>(
+      "cuDevSmResourceSplitByCount");
+  auto gen_desc = driver_fn<CUresult (*)(CUdevResourceDesc*, CUdevResource*, unsigned int)>("cuDevResourceGenerateDesc");
+  auto ctx_create = driver_fn<CUresult (*)(CUgreenCtx*, CUdevResourceDesc, CUdevice, unsigned int)>("cuGreenCtxCreate");
+  auto ctx_destroy = driver_fn<CUresult (*)(CUgreenCtx)>("cuGreenCtxDestroy");
+  auto stream_create = driver_fn<CUresult (*)(CUstream*, CUgreenCtx, unsigned int, int)>("cuGreenCtxStreamCreate");
+  auto dev_get = driver_fn<CUresult (*)(CUdevice*, int)>("cuDeviceGet");
+  if (!get_res || !split || !gen_desc || !ctx_create || !ctx_destroy || !stream_create || !dev_get) return ADIT_E_UNSUPPORTED;
+  CUdevice dev;
+  if (dev_get(&dev, device) != CUDA_SUCCESS) return ADIT_E_CUDA;
+  CUdevResource all, part, rest;
+  if (get_res(dev, &all, CU_DEV_RESOURCE_TYPE_SM) != CUDA_SUCCESS) return ADIT_E_UNSUPPORTED;
+  if ((unsigned)sm_count > all.sm.smCount) return ADIT_E_CAPACITY;
+  unsigned int groups = 1;
+  // one group of at least sm_count SMs (the driver rounds up to its granularity); the remainder is not used here
+  if (split(&part, &groups, &all, &rest, 0, (unsigned)sm_count) != CUDA_SUCCESS || groups != 1) return ADIT_E_UNSUPPORTED;
+  CUdevResourceDesc desc;
+  if (gen_desc(&desc, &part, 1) != CUDA_SUCCESS) return ADIT_E_CUDA;
+  adit_green_stream* g = new (std::nothrow) adit_green_stream();
+  if (!g) return ADIT_E_INVALID;
+  g->device = device; g->sm_count = (int)part.sm.smCount; g->stream = nullptr;
+  if (ctx_create(&g->ctx, desc, dev, CU_GREEN_CTX_DEFAULT_STREAM) != CUDA_SUCCESS) { delete g; return ADIT_E_CUDA; }
+  if (stream_create(&g->stream, g->ctx, CU_STREAM_NON_BLOCKING, 0) != CUDA_SUCCESS) { ctx_destroy(g->ctx); delete g; return ADIT_E_CUDA; }
+  *out = g;
+  return ADIT_OK;
+}
+extern "C" void* adit_green_stream_handle(adit_green_stream* g) { return g ? (void*)g->stream : nullptr; }
+extern "C" int adit_green_stream_sm_count(adit_green_stream* g) { return g ? g->sm_count : 0; }
+extern "C" int adit_green_stream_destroy(adit_green_stream* g) {
+  if (!g) return ADIT_OK;
+  cudaSetDevice(g->device);
+  if (g->stream) { cudaStreamSynchronize((cudaStream_t)g->stream); cudaStreamDestroy((cudaStream_t)g->stream); }
+  auto ctx_destroy = driver_fn<CUresult (*)(CUgreenCtx)>("cuGreenCtxDestroy");
+  if (ctx_destroy) ctx_destroy(g->ctx);
+  delete g;
+  return ADIT_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
 // Background GEMM load (stand-in for the VLM stage on the other stream)
 // ---------------------------------------------------------------------------------------------
 struct adit_bg_gemm {

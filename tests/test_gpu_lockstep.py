@@ -44,3 +44,42 @@ def test_locksteps_on_two_streams_match_direct_calls():
         assert max(v0, a0) < min(v1, a1)
     stages.close()
     eng.close()
+
+
+def test_green_stream_confines_a_kernel_that_asks_for_the_whole_chip():
+    """A stream on a green context (paper section 4.1.2: the VLM stream restricted to a number of SMs in multiples of 8):
+    the stand-in GEMM launched with its full grid takes about as long as with its grid capped to that many SMs, and
+    much longer than on the whole chip; the partition is what was asked for, rounded up to the driver's granularity."""
+    import torch
+    from paper_2609_12075_b200 import build
+    build.build()
+    from paper_2609_12075_b200 import adit
+
+    def per_launch_us(stream, g, cap):
+        g.launch(3, cap, stream)
+        stream.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        g.launch(10, cap, stream)
+        e1.record(stream)
+        stream.synchronize()
+        return e0.elapsed_time(e1) * 100.0
+
+    g = adit.BackgroundGemm(8192, 2048, 2048)
+    plain = torch.cuda.Stream()
+    full, capped = per_launch_us(plain, g, 0), per_launch_us(plain, g, 24)
+    try:
+        gs = adit.GreenStream(20)
+    except adit.AditError as e:
+        if e.code == adit.E_UNSUPPORTED:
+            pytest.skip("no green contexts on this driver")
+        raise
+    assert gs.sm_count >= 20 and gs.sm_count % 8 == 0 and gs.sm_count <= 32
+    confined = per_launch_us(gs.stream, g, 0)
+    gs.close()
+    g.close()
+    assert confined > 2.5 * full            # (24 of 148 SMs: about six times the whole-chip time)
+    assert 0.6 * capped < confined * gs.sm_count / 24 < 1.8 * capped
+    with pytest.raises(adit.AditError) as e:
+        adit.GreenStream(100000)
+    assert e.value.code == adit.E_CAPACITY
