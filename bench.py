@@ -414,6 +414,27 @@ def run_ours(args):
                                  "ms_p99": float(np.percentile(l2, 99)), "ms_mean": float(l2.mean()),
                                  "chunks_per_s": wl.batch / (float(l2.mean()) * 1e-3), "roofline_step": roof}
             del bsets
+        # hidden-state hand-over (the expert projects the prefix K/V itself, once per call): the projection alone, for the
+        # batch-1 and batch-32 prefixes, from hidden states of width 2048
+        big.load_prefix_projection(W.make_prefix_projection(cfg, base.seed, 2048))
+        for name in ("c2", "c4"):
+            wl = WORKLOADS[name](with_kv=False) if name != "c2" else base
+            hid = [torch.from_numpy(W.make_prefix_hidden(wl.seed, b, int(p), 2048)).to(torch.bfloat16).to(dev) for b, p in enumerate(wl.prefix_len)]
+            caches = [torch.zeros((cfg.n_layers, 2, cfg.n_kv_heads, 1024, cfg.head_dim), dtype=torch.bfloat16, device=dev) for _ in hid]
+            with torch.cuda.stream(stream):
+                for i in range(3):
+                    big.project_prefix(hid, wl.prefix_len, caches, stream=stream)
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(stream)
+                for i in range(20):
+                    big.project_prefix(hid, wl.prefix_len, caches, stream=stream)
+                e1.record(stream)
+                stream.synchronize()
+            ms = e0.elapsed_time(e1) / 20
+            flops = 2.0 * float(np.sum(wl.prefix_len)) * 2048 * (2 * cfg.n_layers * cfg.n_kv_heads * cfg.head_dim)
+            by_workload[f"{name}_prefix_projection"] = {"batch": int(len(hid)), "hidden_dim": 2048, "ms": ms, "tflops": flops / (ms * 1e-3) / 1e12,
+                                                        "launches": int(len(hid))}
+            del hid, caches
         assert big.poll_status() == 0
         big.close()
         # the same call as one persistent kernel (opt-in path), for the record

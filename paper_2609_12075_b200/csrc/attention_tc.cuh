@@ -31,12 +31,16 @@ namespace adit {
 namespace attn {
 
 constexpr int TC_ROWS = 128;
-constexpr int TC_LOADERS = 64;   // threads per operand that help to stage a key split's output (warps 4-5, 6-7); thread 0 of each group issues the operand's copies
-constexpr int TC_THREADS = 320;  // warps 0-3 softmax, 4-7 loaders, 8 issuer of Q K^T (+ TMEM owner), 9 issuer of P V
+// warps 0-7 softmax (warps w and w + 4 share 32 query rows and take one half of a key block's columns each), 8 issuer of
+// Q K^T (+ TMEM owner), 9 issuer of P V, 10 K copies, 11 V copies
+constexpr int TC_THREADS = 384;
 
 template <int DH>
 constexpr size_t attn_tc_smem_bytes() {
-  return (size_t)TC_ROWS * DH * 2 + 2 * 2 * (size_t)KEY_BLOCK * DH * 2 + 2 * (size_t)TC_ROWS * KEY_BLOCK * 2 + 1024;
+  // Q tile + two K and two V stages + two P buffers.  The dynamic array is declared 1024-byte aligned, so it starts at
+  // the first such offset behind the kernel's static shared memory (at most 3 KB: with head_dim 256 the sum is
+  // exactly the 227 KB a block may have); smaller head dimensions keep a kilobyte of slack for a run-time round-up.
+  return (size_t)TC_ROWS * DH * 2 + 2 * 2 * (size_t)KEY_BLOCK * DH * 2 + 2 * (size_t)TC_ROWS * KEY_BLOCK * 2 + (DH >= 256 ? 0 : 1024);
 }
 
 __device__ __forceinline__ float ex2(float x) {
@@ -58,8 +62,11 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
                                                                 const PrefixTable* __restrict__ ptp) {
   constexpr int KV_BYTES = KEY_BLOCK * DH * 2;
   constexpr int Q_BYTES = TC_ROWS * DH * 2;
-  extern __shared__ uint8_t smem_raw[];
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t k_full[2], v_full[2], k_empty[2], v_empty[2], s_full[2], s_empty[2], p_full[2], pv_done[2], q_full, o_done;
+  __shared__ __align__(8) uint64_t pair_bar[4];  // hand-shake of the two softmax warps that share 32 rows
+  __shared__ float xch_max[2][2][TC_ROWS];       // [block parity][column half][row]: half-row maxima (and, after the
+                                                 // last block, the half-row sums in the buffer of the other parity)
   __shared__ uint32_t tmem_base_smem;
   __shared__ volatile int abort_flag;
 
@@ -70,6 +77,10 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
   if (dbg && threadIdx.x == 0) dbg[0] = ptx::globaltimer_ns();
   unsigned long long* const dlog = (INSTR && a.dbg && blockIdx.x == 0) ? a.dbg + 8192 : nullptr;  // per-key-block log of block 0
   uint8_t* base = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  if (DH >= 256 && base != smem_raw) {  // (no slack at this size: never expected, and nothing has been touched yet)
+    if (threadIdx.x == 0 && a.status) atomicExch(a.status, -5);
+    return;
+  }
   uint8_t* sQ = base;                       // DH / 64 boxes [128 rows][64 ch]
   uint8_t* sK = sQ + Q_BYTES;               // 2 stages x DH / 64 boxes [64 keys][64 ch]
   uint8_t* sV = sK + 2 * KV_BYTES;          // same
@@ -92,10 +103,11 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
       ptx::mbar_init(&k_empty[s], 1);
       ptx::mbar_init(&v_empty[s], 1);
       ptx::mbar_init(&s_full[s], 1);
-      ptx::mbar_init(&s_empty[s], 4);  // one arrival per softmax warp (128 separate arrivals on one barrier word are slow)
-      ptx::mbar_init(&p_full[s], 4);
+      ptx::mbar_init(&s_empty[s], 8);  // one arrival per softmax warp (separate arrivals of every thread on one barrier word are slow)
+      ptx::mbar_init(&p_full[s], 8);
       ptx::mbar_init(&pv_done[s], 1);
     }
+    for (int w = 0; w < 4; ++w) ptx::mbar_init(&pair_bar[w], 2);
     ptx::mbar_init(&q_full, 1);
     ptx::mbar_init(&o_done, 1);  // all P V products of a work item complete (once per item: no parity doubt for early waiters)
     if (QTMA) ptx::prefetch_tensormap(&map_q);
@@ -115,12 +127,13 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
   // The prefix caches do not depend on the preceding kernel (only Q and the suffix K/V do): the loader
   // warps start on key blocks that lie wholly in the prefix right away and wait for the preceding grid only
   // when they first need a suffix row; every other warp waits once it has worked out its first work item.
-  const bool is_loader = (threadIdx.x >> 5) >= 4 && (threadIdx.x >> 5) < 8;
+  const bool is_loader = (threadIdx.x >> 5) >= 10;
   bool waited = false;
 
   // Barrier phases run on across work items: these counters are kept per role.
   uint32_t kv_cnt = 0;   // key blocks processed so far by this role (block n uses stage, S, P buffer and barriers n & 1)
   uint32_t q_cnt = 0;    // query tiles loaded so far
+  uint32_t pair_cnt = 0; // hand-shakes of this softmax warp with its partner so far
   bool ok = true;
 
   for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
@@ -174,13 +187,13 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
     }
     if (dbg && threadIdx.x == 0 && item == (int)blockIdx.x) dbg[2] = ptx::globaltimer_ns();
 
-    if (warp >= 4 && warp < 8) {
-      // ------------------------------ K loaders (warps 4-5) and V loaders (warps 6-7) ------------------------------
-      const int which = warp >= 6 ? 1 : 0;
+    if (warp >= 10) {
+      // ------------------------------ K copies (warp 10) and V copies (warp 11) ------------------------------
+      const int which = warp == 11 ? 1 : 0;
       uint64_t* empty_bar = which ? v_empty : k_empty;
       uint64_t* full_bar = which ? v_full : k_full;
       uint8_t* ring = which ? sV : sK;
-      if (tid == (which ? 192 : 128)) {
+      if (lane == 0) {
         // one thread per operand issues the copies: dh / 64 boxes of 64 keys x 64 channels per block
         const int plane = (a.layer * 2 + which) * a.n_kv_heads + kvh;
         const CUtensorMap* pm = a.kv_maps + b;
@@ -203,42 +216,11 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
             for (int j = 0; j < DH / 64; ++j)
               ptx::tma_load_2d(dst + j * (KEY_BLOCK * 128), &map_sfx, (which ? v_off : k_off) + kvh * DH + j * 64, rowg, &full_bar[s]);
           }
-          if (dbg && tid == 128 && item == (int)blockIdx.x && i < 2) dbg[3 + i] = ptx::globaltimer_ns();
-          if (dlog && tid == 128 && item == 0 && i < 32) dlog[i * 4 + 0] = ptx::globaltimer_ns();
+          if (dbg && which == 0 && item == (int)blockIdx.x && i < 2) dbg[3 + i] = ptx::globaltimer_ns();
+          if (dlog && which == 0 && item == 0 && i < 32) dlog[i * 4 + 0] = ptx::globaltimer_ns();
         }
+        if (!ok) { if (a.status) atomicExch(a.status, -6); abort_flag = 1; }
       }
-      ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
-      if (!waited && PARTIAL) { ptx::pdl_wait_prior_grids(); waited = true; }  // (before this warp writes partial outputs)
-      // Their loads done, the loader warps help to stage a key split's unnormalised output: warp w can read the same
-      // TMEM lanes as softmax warp w - 4, and takes the upper half of the channels.
-      if (PARTIAL && nb > 0 && ok) {
-        // (the K loaders run several blocks ahead of the P V products: they wait on the per-item barrier, whose
-        // parity cannot be mistaken, not on the per-block ones)
-        int okp = 1;
-        if (lane == 0) okp = ptx::mbar_wait(&o_done, q_cnt & 1) ? 1 : 0;
-        okp = __shfl_sync(0xffffffffu, okp, 0);
-        if (!okp) ok = false;
-        for (int spin = 0; ok && spin < 4096 && !ptx::mbar_try_wait(&o_done, q_cnt & 1); ++spin) {}
-        ptx::tc_fence_after();
-        if (ok) {
-          const int srow_i = (warp & 3) * 32 + lane;
-          const uint32_t la = (uint32_t)((warp & 3) * 32) << 16;
-          uint8_t* srow = sK + (size_t)srow_i * (DH * 2 + 16);
-#pragma unroll 1
-          for (int c0 = DH / 2; c0 < DH; c0 += 32) {
-            float o[32];
-            ptx::tmem_ld_32x32(tm_o + c0 + la, o);
-            ptx::tmem_ld_wait();
-#pragma unroll
-            for (int j = 0; j < 32; j += 8)
-              *reinterpret_cast<uint4*>(srow + (c0 + j) * 2) =
-                  make_uint4(pack_bf16(o[j], o[j + 1]), pack_bf16(o[j + 2], o[j + 3]), pack_bf16(o[j + 4], o[j + 5]),
-                             pack_bf16(o[j + 6], o[j + 7]));
-          }
-          ptx::tc_fence_before();
-        }
-      }
-      if (!ok && lane == 0) { if (a.status) atomicExch(a.status, -6); abort_flag = 1; }
       kv_cnt += nb;
     } else if (warp == 8) {
       // ------------------------------ issuer of S = Q K^T ------------------------------
@@ -247,17 +229,21 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
       // the K stages and the two S buffers allow.
       if (lane == 0) {
         const uint32_t idesc_s = ptx::idesc_bf16_f32(TC_ROWS, KEY_BLOCK);
+        const uint32_t desc_hi = ptx::smem_desc_hi_sw128();
+        const uint32_t q_lo0 = ptx::smem_desc_lo(ptx::smem_u32(sQ)), k_lo0 = ptx::smem_desc_lo(ptx::smem_u32(sK));
         if (nb > 0 && QTMA && !ptx::mbar_wait(&q_full, q_cnt & 1)) ok = false;
         for (int i = 0; i < nb && ok; ++i) {
           const uint32_t n = kv_cnt + i;
           const int s = n & 1;
           if (!ptx::mbar_wait(&k_full[s], (n >> 1) & 1) || !ptx::mbar_wait(&s_empty[s], ((n >> 1) & 1) ^ 1)) { ok = false; break; }
           ptx::tc_fence_after();
-          const uint32_t qa = ptx::smem_u32(sQ), ka = ptx::smem_u32(sK + s * KV_BYTES);
+          // head_dim / 64 groups of four products: descriptor halves in registers, one instruction sequence per group
+          // (this thread's own instruction latencies are what a key block's scores cost)
+          const uint32_t k_lo = k_lo0 + (uint32_t)s * (KV_BYTES >> 4);
 #pragma unroll
-          for (int ks = 0; ks < DH / 16; ++ks)
-            ptx::umma_f16(tm_s + s * KEY_BLOCK, ptx::smem_desc_sw128(qa + (ks >> 2) * (TC_ROWS * 128) + (ks & 3) * 32),
-                          ptx::smem_desc_sw128(ka + (ks >> 2) * (KEY_BLOCK * 128) + (ks & 3) * 32), idesc_s, ks > 0);
+          for (int j = 0; j < DH / 64; ++j)
+            ptx::umma_kblock_f16(tm_s + s * KEY_BLOCK, q_lo0 + j * (TC_ROWS * 128 >> 4), k_lo + j * (KEY_BLOCK * 128 >> 4), desc_hi, idesc_s,
+                                 j > 0 ? 1u : 0u);
           ptx::umma_commit(&s_full[s]);
           ptx::umma_commit(&k_empty[s]);  // the K stage is free as soon as these products have read it
         }
@@ -286,9 +272,16 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
       }
       kv_cnt += nb;
     } else {
-      // ------------------------------ softmax / output (warps 0-3, thread = query row) ------------------------------
-      const int row = tid;  // 0..127, also the TMEM lane
-      const uint32_t lane_addr = (uint32_t)(warp * 32) << 16;
+      // ------------------------------ softmax / output (warps 0-7) ------------------------------
+      // Thread = (query row, column half): warps w and w + 4 can both read the TMEM lanes of rows 32 w .. 32 w + 31 and
+      // take columns [0, 32) and [32, 64) of every key block (and the lower / upper half of the output channels).  With
+      // one warp per scheduler the per-block latencies (barrier tests, tensor-memory loads) lay bare; two warps hide them
+      // for each other.  The row maximum is the only thing the halves have to agree on: they exchange their half-row
+      // maxima through shared memory once per block and then take identical decisions.
+      const int half = warp >> 2, wq = warp & 3;
+      const int row = wq * 32 + lane;  // 0..127, also the TMEM lane
+      const uint32_t lane_addr = (uint32_t)(wq * 32) << 16;
+      constexpr int HB = KEY_BLOCK / 2;  // columns of a key block per thread
       // Wait of a whole warp: one non-blocking test by every lane when the phase is already complete (a barrier
       // instruction costs over a hundred cycles), otherwise lane 0 waits with the time limit and the others follow.
       auto warp_wait = [&](uint64_t* bar, uint32_t parity) -> bool {
@@ -300,6 +293,15 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
         for (int spin = 0; spin < 4096 && !ptx::mbar_try_wait(bar, parity); ++spin) {}
         return true;
       };
+      // Bounded hand-shake with the warp that shares this warp's rows (an mbarrier, not bar.sync: a warp that gave up
+      // on a wait must not strand its partner).  Orders this warp's shared-memory writes before the partner's reads.
+      auto pair_sync = [&]() -> bool {
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(&pair_bar[wq]);
+        const bool okp = warp_wait(&pair_bar[wq], pair_cnt & 1);
+        ++pair_cnt;
+        return okp;
+      };
       float m_ref = -INFINITY, l = 0.f;
       for (int i = 0; i < nb && ok; ++i) {
         const uint32_t n = kv_cnt + i;
@@ -308,9 +310,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
         ptx::tc_fence_after();
         if (dbg && tid == 0 && item == (int)blockIdx.x && i < 2) dbg[5 + 2 * i] = ptx::globaltimer_ns();
         if (dlog && tid == 0 && item == 0 && i < 32) dlog[i * 4 + 1] = ptx::globaltimer_ns();
-        float sc[64];
-        ptx::tmem_ld_32x32(tm_s + s * KEY_BLOCK + lane_addr, sc);
-        ptx::tmem_ld_32x32(tm_s + s * KEY_BLOCK + 32 + lane_addr, sc + 32);
+        float sc[HB];
+        ptx::tmem_ld_32x32(tm_s + s * KEY_BLOCK + half * HB + lane_addr, sc);
         ptx::tmem_ld_wait();
         ptx::tc_fence_before();
         __syncwarp();
@@ -322,25 +323,28 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
         const int nvalid = blk < npb ? min(KEY_BLOCK, plen - blk * KEY_BLOCK) : min(KEY_BLOCK, a.n_tokens - (blk - npb) * KEY_BLOCK);
         if (nvalid < KEY_BLOCK) {
 #pragma unroll
-          for (int j = 0; j < 64; ++j)
-            if (j >= nvalid) sc[j] = -INFINITY;
+          for (int j = 0; j < HB; ++j)
+            if (half * HB + j >= nvalid) sc[j] = -INFINITY;
         }
         // variant: the state token's rows (token 0 of the request: rows 0 .. G-1 of row tile 0) see, of the suffix,
         // the state token's own key only
         if (a.state_mask && rt * TC_ROWS + row < G && blk >= npb) {
-          const int first = (blk - npb) * KEY_BLOCK;
+          const int first = (blk - npb) * KEY_BLOCK + half * HB;
 #pragma unroll
-          for (int j = 0; j < 64; ++j)
+          for (int j = 0; j < HB; ++j)
             if (first + j > 0) sc[j] = -INFINITY;
         }
-        // (four independent chains: a single thread per scheduler cannot hide the latency of one long chain)
+        // (four independent chains: a thread cannot hide the latency of one long chain)
         float mx[4] = {sc[0], sc[1], sc[2], sc[3]};
 #pragma unroll
-        for (int j = 4; j < 64; j += 4) {
+        for (int j = 4; j < HB; j += 4) {
           mx[0] = fmaxf(mx[0], sc[j]); mx[1] = fmaxf(mx[1], sc[j + 1]);
           mx[2] = fmaxf(mx[2], sc[j + 2]); mx[3] = fmaxf(mx[3], sc[j + 3]);
         }
-        const float mraw = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+        const float mhalf = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+        xch_max[i & 1][half][row] = mhalf;
+        if (!pair_sync()) { ok = false; break; }
+        const float mraw = fmaxf(mhalf, xch_max[i & 1][half ^ 1][row]);
         const float mb = mraw * a.scale_log2;
         // the reference maximum only moves when it would otherwise be exceeded by more than 2^8
         float corr = 1.f;
@@ -350,13 +354,14 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
           m_ref = mb;
           l *= corr;
         }
-        // O may only be rescaled once the previous P V has completed (rare after the first blocks)
+        // O may only be rescaled once the previous P V has completed (rare after the first blocks); each half
+        // rescales its half of the channels (both warps of a pair see the same rows, hence the same decision)
         if (i > 0 && __any_sync(0xffffffffu, grow)) {
           const uint32_t q = n - 1;
           if (!warp_wait(&pv_done[q & 1], (q >> 1) & 1)) { ok = false; break; }
           ptx::tc_fence_after();
 #pragma unroll 1
-          for (int c0 = 0; c0 < DH; c0 += 32) {
+          for (int c0 = half * (DH / 2); c0 < (half + 1) * (DH / 2); c0 += 32) {
             float o[32];
             ptx::tmem_ld_32x32(tm_o + c0 + lane_addr, o);
             ptx::tmem_ld_wait();
@@ -376,10 +381,10 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
         // (a key range whose keys are all masked for this row leaves the reference maximum at -inf: subtract 0 then,
         // so that the probabilities are exp2(-inf) = 0 and not NaN)
         const float m_sub = m_ref == -INFINITY ? 0.f : m_ref;
-        // probabilities -> bf16 -> shared memory (row = 128 bytes = 8 swizzled chunks)
+        // probabilities -> bf16 -> shared memory (row = 128 bytes = 8 swizzled chunks, four of them this thread's)
         float rs[4] = {0.f, 0.f, 0.f, 0.f};  // partial row sums, added up in a fixed order
 #pragma unroll
-        for (int c = 0; c < 8; ++c) {
+        for (int c = 0; c < HB / 8; ++c) {
           uint32_t w[4];
 #pragma unroll
           for (int q = 0; q < 4; ++q) {
@@ -387,7 +392,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
             rs[q] += p0 + p1;
             w[q] = pack_bf16(p0, p1);
           }
-          *reinterpret_cast<uint4*>(sPn + swz(row, c)) = make_uint4(w[0], w[1], w[2], w[3]);
+          *reinterpret_cast<uint4*>(sPn + swz(row, half * (HB / 8) + c)) = make_uint4(w[0], w[1], w[2], w[3]);
         }
         l += (rs[0] + rs[1]) + (rs[2] + rs[3]);
         ptx::fence_proxy_async();
@@ -397,6 +402,13 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
         if (dbg && tid == 0 && item == (int)blockIdx.x && i < 2) dbg[6 + 2 * i] = ptx::globaltimer_ns();
         if (dlog && tid == 0 && item == 0 && i < 32) dlog[i * 4 + 2] = ptx::globaltimer_ns();
       }
+      // the row sum: this half's part plus the partner's, lower half first
+      if (ok && nb > 0) {
+        // (the buffer of parity nb & 1 was last read one hand-shake ago)
+        xch_max[nb & 1][half][row] = l;
+        if (!pair_sync()) ok = false;
+        l = xch_max[nb & 1][0][row] + xch_max[nb & 1][1][row];
+      }
       // ---- output ----
       if (ok && nb > 0) {
         const uint32_t q = kv_cnt + nb - 1;
@@ -404,16 +416,15 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
         ptx::tc_fence_after();
       }
       if (dbg && tid == 0 && item == (int)blockIdx.x) dbg[9] = ptx::globaltimer_ns();
-      // Each thread owns one row, so direct stores would touch 32 different lines per instruction: the
+      // Each thread owns half a row, so direct stores would touch 32 different lines per instruction: the
       // rows are staged in shared memory (the K/V/P buffers are free now) and written out by the whole block
       // with contiguous 16-byte stores.
       const int gr = rt * TC_ROWS + row;
       const bool row_ok = gr < R;
       const float inv = PARTIAL ? 1.0f : 1.0f / l;
       uint8_t* srow = stage + (size_t)row * STAGE_STRIDE;
-      const int c_end = (PARTIAL && nb > 0 && DH >= 64) ? DH / 2 : DH;  // (the loader warps stage the other half)
 #pragma unroll 1
-      for (int c0 = 0; c0 < c_end; c0 += 32) {
+      for (int c0 = half * (DH / 2); c0 < (half + 1) * (DH / 2); c0 += 32) {
         float o[32];
         if (nb > 0 && ok) {
           ptx::tmem_ld_32x32(tm_o + c0 + lane_addr, o);
@@ -429,7 +440,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
               make_uint4(pack_bf16(o[j] * inv, o[j + 1] * inv), pack_bf16(o[j + 2] * inv, o[j + 3] * inv),
                          pack_bf16(o[j + 4] * inv, o[j + 5] * inv), pack_bf16(o[j + 6] * inv, o[j + 7] * inv));
       }
-      if (PARTIAL && row_ok) {
+      if (PARTIAL && row_ok && half == 0) {
         const int tok = gr / G, hq = kvh * G + gr % G;
         const int64_t qrow = (tok0 + tok) * a.n_q_heads + hq;
         const int64_t n_qrows = (int64_t)a.batch * a.n_tokens * a.n_q_heads;
