@@ -4,11 +4,15 @@
 // r / G with query head kvh * G + r % G - against a range of 64-key blocks of the key list
 // [prefix 0..P_b) ++ [suffix 0..N).  Per key block:
 //   S = Q K^T        tcgen05.mma, M = 128 rows, N = 64 keys, K = head_dim; S lives in TMEM (2 buffers)
-//   softmax          4 warps, one thread per query row: the row's 64 scores come out of TMEM with
-//                    tcgen05.ld, so row max and row sum are plain per-thread loops (no shuffles);
-//                    exp2 with log2(e)/sqrt(dh) folded into the scale; P goes to shared memory as bf16
-//   O += P V         tcgen05.mma, M = 128, N = head_dim, K = 64 keys; V is used as stored ([key][channel],
-//                    an MN-major operand), O accumulates in TMEM
+//   softmax          8 warps: warps w and w + 4 share the 32 rows of TMEM lane quadrant w and take one half of the
+//                    block's 64 columns each, so that every scheduler has two warps to hide the per-block latencies
+//                    (barrier tests, tcgen05.ld) of the other; a thread's 32 scores come out of TMEM with
+//                    tcgen05.ld, row max and row sum are plain per-thread loops, the two half-row maxima are
+//                    exchanged through shared memory (bounded mbarrier hand-shake) and both threads then take the
+//                    same decisions; exp2 with log2(e)/sqrt(dh) folded into the scale; P goes back to TENSOR
+//                    memory as bf16 pairs (tcgen05.st): no shared-memory round trip, no proxy fence
+//   O += P V         tcgen05.mma with the A operand (P) in tensor memory, M = 128, N = head_dim, K = 64 keys; V is
+//                    used as stored ([key][channel], an MN-major operand), O accumulates in TMEM
 // O is only rescaled when a row's running maximum grows by more than 2^8 (the reference maximum is kept
 // otherwise), which keeps the TMEM read-modify-write off the common path.
 //
@@ -17,9 +21,11 @@
 // both come in by TMA (cp.async.bulk.tensor, 128-byte swizzle = the layout the MMA descriptors expect), issued by
 // one thread per operand.  The prefix cache is described by a per-request tensor map whose row extent is the prefix
 // length: rows at or beyond it are never read (the copy engine writes zeros), and their scores are masked to -inf.
-// The K and V rings (two stages each) are released separately - a K stage as soon as its Q K^T has
-// completed, a V stage after its P V - and P is double-buffered, so the softmax of block n only
-// depends on the tensor core through S(n) and, when a row maximum forces a rescale of O, P V(n - 1).
+// The K ring (two stages) and the V ring (three: V is needed last in a block's chain, and its ring has to cover the
+// copies' latency of about a microsecond) are released separately - a K stage as soon as its Q K^T has completed, a V
+// stage after its P V - and P is double-buffered, so the softmax of block n only depends on the tensor core through
+// S(n), P V(n - 2) and, when a row maximum forces a rescale of O, P V(n - 1).  Tensor memory: O 256 columns, S 2 x 64,
+// P 2 x 32.  Shared memory at head_dim 256: Q 64 KB + 5 stages of 32 KB + 3 KB of barriers = the 227 KB of a block.
 // Every mbarrier wait is bounded.  With more than one key split the block writes its unnormalised
 // partial (O as bf16, m, l) and the merge kernel combines the splits in fixed order.
 #pragma once
@@ -34,13 +40,15 @@ constexpr int TC_ROWS = 128;
 // warps 0-7 softmax (warps w and w + 4 share 32 query rows and take one half of a key block's columns each), 8 issuer of
 // Q K^T (+ TMEM owner), 9 issuer of P V, 10 K copies, 11 V copies
 constexpr int TC_THREADS = 384;
+constexpr int V_STAGES = 3;  // V is consumed last in a key block's chain: its ring has to cover the copies' latency
 
 template <int DH>
 constexpr size_t attn_tc_smem_bytes() {
-  // Q tile + two K and two V stages + two P buffers.  The dynamic array is declared 1024-byte aligned, so it starts at
-  // the first such offset behind the kernel's static shared memory (at most 3 KB: with head_dim 256 the sum is
-  // exactly the 227 KB a block may have); smaller head dimensions keep a kilobyte of slack for a run-time round-up.
-  return (size_t)TC_ROWS * DH * 2 + 2 * 2 * (size_t)KEY_BLOCK * DH * 2 + 2 * (size_t)TC_ROWS * KEY_BLOCK * 2 + (DH >= 256 ? 0 : 1024);
+  // Q tile + two K stages + three V stages (the probabilities live in tensor memory).  The dynamic array is declared
+  // 1024-byte aligned, so it starts at the first such offset behind the kernel's static shared memory (at most 3 KB:
+  // with head_dim 256 the sum is exactly the 227 KB a block may have); smaller head dimensions keep a kilobyte of
+  // slack for a run-time round-up.
+  return (size_t)TC_ROWS * DH * 2 + (2 + V_STAGES) * (size_t)KEY_BLOCK * DH * 2 + (DH >= 256 ? 0 : 1024);
 }
 
 __device__ __forceinline__ float ex2(float x) {
@@ -63,7 +71,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
   constexpr int KV_BYTES = KEY_BLOCK * DH * 2;
   constexpr int Q_BYTES = TC_ROWS * DH * 2;
   extern __shared__ __align__(1024) uint8_t smem_raw[];
-  __shared__ __align__(8) uint64_t k_full[2], v_full[2], k_empty[2], v_empty[2], s_full[2], s_empty[2], p_full[2], pv_done[2], q_full, o_done;
+  __shared__ __align__(8) uint64_t k_full[2], v_full[V_STAGES], k_empty[2], v_empty[V_STAGES], s_full[2], s_empty[2], p_full[2], pv_done[2], q_full, o_done;
   __shared__ __align__(8) uint64_t pair_bar[4];  // hand-shake of the two softmax warps that share 32 rows
   __shared__ float xch_max[2][2][TC_ROWS];       // [block parity][column half][row]: half-row maxima (and, after the
                                                  // last block, the half-row sums in the buffer of the other parity)
@@ -83,10 +91,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
   }
   uint8_t* sQ = base;                       // DH / 64 boxes [128 rows][64 ch]
   uint8_t* sK = sQ + Q_BYTES;               // 2 stages x DH / 64 boxes [64 keys][64 ch]
-  uint8_t* sV = sK + 2 * KV_BYTES;          // same
-  uint8_t* sP = sV + 2 * KV_BYTES;          // 2 x [128 rows][64 keys]
-  constexpr int P_BYTES = TC_ROWS * KEY_BLOCK * 2;
-  uint8_t* stage = sK;                      // output staging, aliases sK..sP once the products are done
+  uint8_t* sV = sK + 2 * KV_BYTES;          // V_STAGES stages, same boxes
+  uint8_t* stage = sK;                      // output staging, aliases sK, sV once the products are done
   constexpr int STAGE_STRIDE = DH * 2 + 16; // bf16 row + 16 bytes against bank conflicts
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const PrefixTable& pt = *ptp;
@@ -99,14 +105,13 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
   if (tid == 0) {
     for (int s = 0; s < 2; ++s) {
       ptx::mbar_init(&k_full[s], 1);  // the loading thread's expect-tx arrival; the copies count the bytes
-      ptx::mbar_init(&v_full[s], 1);
       ptx::mbar_init(&k_empty[s], 1);
-      ptx::mbar_init(&v_empty[s], 1);
       ptx::mbar_init(&s_full[s], 1);
       ptx::mbar_init(&s_empty[s], 8);  // one arrival per softmax warp (separate arrivals of every thread on one barrier word are slow)
       ptx::mbar_init(&p_full[s], 8);
       ptx::mbar_init(&pv_done[s], 1);
     }
+    for (int v = 0; v < V_STAGES; ++v) { ptx::mbar_init(&v_full[v], 1); ptx::mbar_init(&v_empty[v], 1); }
     for (int w = 0; w < 4; ++w) ptx::mbar_init(&pair_bar[w], 2);
     ptx::mbar_init(&q_full, 1);
     ptx::mbar_init(&o_done, 1);  // all P V products of a work item complete (once per item: no parity doubt for early waiters)
@@ -124,6 +129,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
   const uint32_t tmem = tmem_base_smem;
   const uint32_t tm_o = tmem;             // O: DH columns
   const uint32_t tm_s = tmem + 256;       // S: 2 x 64 columns
+  const uint32_t tm_p = tmem + 384;       // P: 2 x 32 columns (bf16 pairs: the A operand of P V, read straight from here)
   // The prefix caches do not depend on the preceding kernel (only Q and the suffix K/V do): the loader
   // warps start on key blocks that lie wholly in the prefix right away and wait for the preceding grid only
   // when they first need a suffix row; every other warp waits once it has worked out its first work item.
@@ -200,8 +206,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
         if (npb > 0 && kb0 < npb) ptx::tensormap_acquire(pm);
         for (int i = 0; i < nb && ok; ++i) {
           const uint32_t n = kv_cnt + i;
-          const int s = n & 1;
-          if (!ptx::mbar_wait(&empty_bar[s], ((n >> 1) & 1) ^ 1)) { ok = false; break; }
+          const int s = which ? (int)(n % V_STAGES) : (int)(n & 1);
+          const uint32_t par = which ? ((n / V_STAGES) & 1) : ((n >> 1) & 1);
+          if (!ptx::mbar_wait(&empty_bar[s], par ^ 1)) { ok = false; break; }
           uint8_t* dst = ring + s * KV_BYTES;
           const int blk = kb0 + i;
           ptx::mbar_arrive_expect_tx(&full_bar[s], KV_BYTES);
@@ -256,15 +263,17 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
         const uint32_t idesc_o = ptx::idesc_bf16_f32(TC_ROWS, DH) | (1u << 16);  // B (= V) is MN-major
         for (int i = 0; i < nb && ok; ++i) {
           const uint32_t n = kv_cnt + i;
-          if (!ptx::mbar_wait(&p_full[n & 1], (n >> 1) & 1) || !ptx::mbar_wait(&v_full[n & 1], (n >> 1) & 1)) { ok = false; break; }
+          const int vs = (int)(n % V_STAGES);
+          if (!ptx::mbar_wait(&v_full[vs], (n / V_STAGES) & 1) || !ptx::mbar_wait_hot(&p_full[n & 1], (n >> 1) & 1)) { ok = false; break; }
           ptx::tc_fence_after();
-          const uint32_t pa = ptx::smem_u32(sP + (n & 1) * P_BYTES), va = ptx::smem_u32(sV + (n & 1) * KV_BYTES);
+          // P is read out of tensor memory (8 columns of bf16 pairs per product), V out of its stage
+          const uint32_t pa = tm_p + (n & 1) * (KEY_BLOCK / 2), va = ptx::smem_u32(sV + vs * KV_BYTES);
 #pragma unroll
           for (int k4 = 0; k4 < KEY_BLOCK / 16; ++k4)
-            ptx::umma_f16(tm_o, ptx::smem_desc_sw128(pa + k4 * 32), ptx::smem_desc_mn_sw128(va + k4 * 16 * 128, KEY_BLOCK * 128),
-                          idesc_o, (i > 0 || k4 > 0) ? 1u : 0u);
+            ptx::umma_f16_ta(tm_o, pa + k4 * 8, ptx::smem_desc_mn_sw128(va + k4 * 16 * 128, KEY_BLOCK * 128), idesc_o,
+                             (i > 0 || k4 > 0) ? 1u : 0u);
           ptx::umma_commit(&pv_done[n & 1]);
-          ptx::umma_commit(&v_empty[n & 1]);
+          ptx::umma_commit(&v_empty[vs]);
           if (i == nb - 1) ptx::umma_commit(&o_done);
           if (dlog && item == 0 && i < 32) dlog[i * 4 + 3] = ptx::globaltimer_ns();
         }
@@ -377,25 +386,24 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
           const uint32_t q = n - 2;
           if (!warp_wait(&pv_done[q & 1], (q >> 1) & 1)) { ok = false; break; }
         }
-        uint8_t* sPn = sP + s * P_BYTES;
         // (a key range whose keys are all masked for this row leaves the reference maximum at -inf: subtract 0 then,
         // so that the probabilities are exp2(-inf) = 0 and not NaN)
         const float m_sub = m_ref == -INFINITY ? 0.f : m_ref;
-        // probabilities -> bf16 -> shared memory (row = 128 bytes = 8 swizzled chunks, four of them this thread's)
+        // probabilities -> bf16 pairs -> tensor memory: this thread's 32 keys are 16 columns of its row (lane)
         float rs[4] = {0.f, 0.f, 0.f, 0.f};  // partial row sums, added up in a fixed order
+        uint32_t pw[HB / 2];
 #pragma unroll
         for (int c = 0; c < HB / 8; ++c) {
-          uint32_t w[4];
 #pragma unroll
           for (int q = 0; q < 4; ++q) {
             const float p0 = ex2(fmaf(sc[c * 8 + 2 * q], a.scale_log2, -m_sub)), p1 = ex2(fmaf(sc[c * 8 + 2 * q + 1], a.scale_log2, -m_sub));
             rs[q] += p0 + p1;
-            w[q] = pack_bf16(p0, p1);
+            pw[c * 4 + q] = pack_bf16(p0, p1);
           }
-          *reinterpret_cast<uint4*>(sPn + swz(row, half * (HB / 8) + c)) = make_uint4(w[0], w[1], w[2], w[3]);
         }
         l += (rs[0] + rs[1]) + (rs[2] + rs[3]);
-        ptx::fence_proxy_async();
+        ptx::tmem_st_32x16(tm_p + s * (KEY_BLOCK / 2) + half * (HB / 2) + lane_addr, pw);
+        ptx::tmem_st_wait();
         ptx::tc_fence_before();
         __syncwarp();
         if (lane == 0) ptx::mbar_arrive(&p_full[s]);
