@@ -25,7 +25,7 @@
 // copies' latency of about a microsecond) are released separately - a K stage as soon as its Q K^T has completed, a V
 // stage after its P V - and P is double-buffered, so the softmax of block n only depends on the tensor core through
 // S(n), P V(n - 2) and, when a row maximum forces a rescale of O, P V(n - 1).  Tensor memory: O 256 columns, S 2 x 64,
-// P 2 x 32.  Shared memory at head_dim 256: Q 64 KB + 5 stages of 32 KB + 3 KB of barriers = the 227 KB of a block.
+// P 3 x 32.  Shared memory at head_dim 256: Q 64 KB + 5 stages of 32 KB + 3 KB of barriers = the 227 KB of a block.
 // Every mbarrier wait is bounded.  With more than one key split the block writes its unnormalised
 // partial (O as bf16, m, l) and the merge kernel combines the splits in fixed order.
 #pragma once
@@ -40,6 +40,7 @@ constexpr int TC_ROWS = 128;
 // warps 0-7 softmax (warps w and w + 4 share 32 query rows and take one half of a key block's columns each), 8 issuer of
 // Q K^T (+ TMEM owner), 9 issuer of P V, 10 K copies, 11 V copies
 constexpr int TC_THREADS = 384;
+constexpr int P_BUFS = 3;    // probability buffers in tensor memory: block n may be written while P V(n - 1), P V(n - 2) are pending
 constexpr int V_STAGES = 3;  // V is consumed last in a key block's chain: its ring has to cover the copies' latency
 
 template <int DH>
@@ -71,7 +72,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
   constexpr int KV_BYTES = KEY_BLOCK * DH * 2;
   constexpr int Q_BYTES = TC_ROWS * DH * 2;
   extern __shared__ __align__(1024) uint8_t smem_raw[];
-  __shared__ __align__(8) uint64_t k_full[2], v_full[V_STAGES], k_empty[2], v_empty[V_STAGES], s_full[2], s_empty[2], p_full[2], pv_done[2], q_full, o_done;
+  __shared__ __align__(8) uint64_t k_full[2], v_full[V_STAGES], k_empty[2], v_empty[V_STAGES], s_full[2], s_empty[2], p_full[P_BUFS], pv_done[P_BUFS], q_full, o_done;
   __shared__ __align__(8) uint64_t pair_bar[4];  // hand-shake of the two softmax warps that share 32 rows
   __shared__ float xch_max[2][2][TC_ROWS];       // [block parity][column half][row]: half-row maxima (and, after the
                                                  // last block, the half-row sums in the buffer of the other parity)
@@ -108,10 +109,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
       ptx::mbar_init(&k_empty[s], 1);
       ptx::mbar_init(&s_full[s], 1);
       ptx::mbar_init(&s_empty[s], 8);  // one arrival per softmax warp (separate arrivals of every thread on one barrier word are slow)
-      ptx::mbar_init(&p_full[s], 8);
-      ptx::mbar_init(&pv_done[s], 1);
     }
     for (int v = 0; v < V_STAGES; ++v) { ptx::mbar_init(&v_full[v], 1); ptx::mbar_init(&v_empty[v], 1); }
+    for (int v = 0; v < P_BUFS; ++v) { ptx::mbar_init(&p_full[v], 8); ptx::mbar_init(&pv_done[v], 1); }
     for (int w = 0; w < 4; ++w) ptx::mbar_init(&pair_bar[w], 2);
     ptx::mbar_init(&q_full, 1);
     ptx::mbar_init(&o_done, 1);  // all P V products of a work item complete (once per item: no parity doubt for early waiters)
@@ -129,7 +129,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
   const uint32_t tmem = tmem_base_smem;
   const uint32_t tm_o = tmem;             // O: DH columns
   const uint32_t tm_s = tmem + 256;       // S: 2 x 64 columns
-  const uint32_t tm_p = tmem + 384;       // P: 2 x 32 columns (bf16 pairs: the A operand of P V, read straight from here)
+  const uint32_t tm_p = tmem + 384;       // P: P_BUFS x 32 columns (bf16 pairs: the A operand of P V, read straight from here)
   // The prefix caches do not depend on the preceding kernel (only Q and the suffix K/V do): the loader
   // warps start on key blocks that lie wholly in the prefix right away and wait for the preceding grid only
   // when they first need a suffix row; every other warp waits once it has worked out its first work item.
@@ -264,15 +264,16 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
         for (int i = 0; i < nb && ok; ++i) {
           const uint32_t n = kv_cnt + i;
           const int vs = (int)(n % V_STAGES);
-          if (!ptx::mbar_wait(&v_full[vs], (n / V_STAGES) & 1) || !ptx::mbar_wait_hot(&p_full[n & 1], (n >> 1) & 1)) { ok = false; break; }
+          const int ps = (int)(n % P_BUFS);
+          if (!ptx::mbar_wait(&v_full[vs], (n / V_STAGES) & 1) || !ptx::mbar_wait_hot(&p_full[ps], (n / P_BUFS) & 1)) { ok = false; break; }
           ptx::tc_fence_after();
           // P is read out of tensor memory (8 columns of bf16 pairs per product), V out of its stage
-          const uint32_t pa = tm_p + (n & 1) * (KEY_BLOCK / 2), va = ptx::smem_u32(sV + vs * KV_BYTES);
+          const uint32_t pa = tm_p + ps * (KEY_BLOCK / 2), va = ptx::smem_u32(sV + vs * KV_BYTES);
 #pragma unroll
           for (int k4 = 0; k4 < KEY_BLOCK / 16; ++k4)
             ptx::umma_f16_ta(tm_o, pa + k4 * 8, ptx::smem_desc_mn_sw128(va + k4 * 16 * 128, KEY_BLOCK * 128), idesc_o,
                              (i > 0 || k4 > 0) ? 1u : 0u);
-          ptx::umma_commit(&pv_done[n & 1]);
+          ptx::umma_commit(&pv_done[ps]);
           ptx::umma_commit(&v_empty[vs]);
           if (i == nb - 1) ptx::umma_commit(&o_done);
           if (dlog && item == 0 && i < 32) dlog[i * 4 + 3] = ptx::globaltimer_ns();
@@ -367,7 +368,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
         // rescales its half of the channels (both warps of a pair see the same rows, hence the same decision)
         if (i > 0 && __any_sync(0xffffffffu, grow)) {
           const uint32_t q = n - 1;
-          if (!warp_wait(&pv_done[q & 1], (q >> 1) & 1)) { ok = false; break; }
+          if (!warp_wait(&pv_done[q % P_BUFS], (q / P_BUFS) & 1)) { ok = false; break; }
           ptx::tc_fence_after();
 #pragma unroll 1
           for (int c0 = half * (DH / 2); c0 < (half + 1) * (DH / 2); c0 += 32) {
@@ -381,10 +382,10 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
           ptx::tmem_st_wait();
           ptx::tc_fence_before();
         }
-        // this block's P buffer was last read by the P V two blocks back
-        if (i >= 2) {
-          const uint32_t q = n - 2;
-          if (!warp_wait(&pv_done[q & 1], (q >> 1) & 1)) { ok = false; break; }
+        // this block's P buffer was last read by the P V three blocks back
+        if (i >= P_BUFS) {
+          const uint32_t q = n - P_BUFS;
+          if (!warp_wait(&pv_done[q % P_BUFS], (q / P_BUFS) & 1)) { ok = false; break; }
         }
         // (a key range whose keys are all masked for this row leaves the reference maximum at -inf: subtract 0 then,
         // so that the probabilities are exp2(-inf) = 0 and not NaN)
@@ -402,11 +403,12 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
           }
         }
         l += (rs[0] + rs[1]) + (rs[2] + rs[3]);
-        ptx::tmem_st_32x16(tm_p + s * (KEY_BLOCK / 2) + half * (HB / 2) + lane_addr, pw);
+        const int ps = (int)(n % P_BUFS);
+        ptx::tmem_st_32x16(tm_p + ps * (KEY_BLOCK / 2) + half * (HB / 2) + lane_addr, pw);
         ptx::tmem_st_wait();
         ptx::tc_fence_before();
         __syncwarp();
-        if (lane == 0) ptx::mbar_arrive(&p_full[s]);
+        if (lane == 0) ptx::mbar_arrive(&p_full[ps]);
         if (dbg && tid == 0 && item == (int)blockIdx.x && i < 2) dbg[6 + 2 * i] = ptx::globaltimer_ns();
         if (dlog && tid == 0 && item == 0 && i < 32) dlog[i * 4 + 2] = ptx::globaltimer_ns();
       }
@@ -420,7 +422,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
       // ---- output ----
       if (ok && nb > 0) {
         const uint32_t q = kv_cnt + nb - 1;
-        if (!warp_wait(&pv_done[q & 1], (q >> 1) & 1)) ok = false;
+        if (!warp_wait(&pv_done[q % P_BUFS], (q / P_BUFS) & 1)) ok = false;
         ptx::tc_fence_after();
       }
       if (dbg && tid == 0 && item == (int)blockIdx.x) dbg[9] = ptx::globaltimer_ns();
