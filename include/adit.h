@@ -283,6 +283,17 @@ const char* adit_strerror(int code);
 int64_t adit_debug_copy(adit_handle* h, const char* name, void* host_dst, size_t nbytes);
 
 /*
+ * adit_debug_gemm_timeout: failure-path test aid for the kernel-per-phase path.  Runs a small projection
+ * in which one thread block is denied one operand copy, so that one of its bounded device-side waits
+ * expires (about two seconds, the kernels' limit), the block records ADIT_E_TIMEOUT in the status word,
+ * waits for its copies in flight, frees its tensor memory and returns; then runs the same projection
+ * untouched.  *first_status = the status word after the first run (ADIT_E_TIMEOUT expected); returns the
+ * status after the second run (ADIT_OK expected) or a host-side error.  No trap, no fault, no unbounded
+ * wait.  Synchronises the stream.  The paper has no counterpart.
+ */
+int adit_debug_gemm_timeout(int device, int* first_status, void* stream);
+
+/*
  * adit_debug_gemm: run the tensor-core projection kernel on its own (test aid): out[n_tok, n_feat]
  * (fp32, device) = A[n_tok, k] W[n_feat, k]^T with bf16 device operands, k a multiple of 64;
  * splits = 0 lets the library choose the k-split, splits = -2 selects the two-SM kernel (pairs of

@@ -255,6 +255,62 @@ extern "C" int adit_debug_gemm(int device, int n_tok, int n_feat, int k, const v
 }
 
 
+// Makes a bounded device-side wait of the projection kernel run out, once, on purpose-built operands: block 0 of a
+// small product (51 tokens x 2560 features x 1024, no k-split: no cluster is involved) never gets the tokens of its
+// third k-block, so its issuing thread's wait on that stage expires after the kernel's two-second limit, the block
+// records ADIT_E_TIMEOUT, lets its copies land, frees its tensor memory and returns like the others.  The same
+// product is then run again untouched.  *first_status receives the status word after the first run (ADIT_E_TIMEOUT
+// expected), the return value is the status after the second (ADIT_OK expected) or a host-side error.
+extern "C" int adit_debug_gemm_timeout(int device, int* first_status, void* stream) {
+  if (!first_status) return ADIT_E_INVALID;
+  if (cudaSetDevice(device) != cudaSuccess) return ADIT_E_CUDA;
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return ADIT_E_CUDA;
+  if (prop.major != 10) return ADIT_E_UNSUPPORTED;
+  if (tc::ensure_smem_attr() != cudaSuccess) return ADIT_E_CUDA;
+  const int n_tok = 51, n_feat = 2560, k = 1024, SM = prop.multiProcessorCount;
+  const tc::GemmPlan p = tc::plan_gemm(n_tok, n_feat, k, false, SM, false);  // (k-split not allowed)
+  if (p.splits != 1) return ADIT_E_UNSUPPORTED;
+  void *a = nullptr, *w = nullptr;
+  float* out = nullptr;
+  int* status = nullptr;
+  const size_t rows_padded = (size_t)p.n_ttiles * p.tile_tok;
+  bool ok = cudaMalloc(&a, (size_t)rows_padded * k * 2) == cudaSuccess && cudaMalloc(&w, (size_t)n_feat * k * 2) == cudaSuccess &&
+            cudaMalloc((void**)&out, rows_padded * n_feat * 4) == cudaSuccess && cudaMalloc((void**)&status, 4) == cudaSuccess;
+  int rc = ADIT_E_CUDA;
+  if (ok) {
+    cudaMemset(a, 0, rows_padded * k * 2);
+    cudaMemset(w, 0, (size_t)n_feat * k * 2);
+    cudaMemset(status, 0, 4);
+    CUtensorMap mw, ma;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (tc::make_map_bf16(&mw, w, n_feat, k, tc::TILE_F) && tc::make_map_bf16(&ma, a, rows_padded, k, p.tile_tok)) {
+      tc::GemmArgs g{};
+      g.n_feat = n_feat; g.n_tok = n_tok; g.epi = EPI_STORE_F32; g.out = out; g.ldo = n_feat; g.status = status;
+      g.debug_withhold = 3;
+      cudaError_t e = tc::launch_gemm(mw, ma, p, false, g, SM, st);
+      if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+      int hs = 0;
+      if (e == cudaSuccess) e = cudaMemcpy(&hs, status, 4, cudaMemcpyDeviceToHost);
+      *first_status = hs;
+      if (e == cudaSuccess) {
+        cudaMemset(status, 0, 4);
+        g.debug_withhold = 0;
+        e = tc::launch_gemm(mw, ma, p, false, g, SM, st);
+        if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+        if (e == cudaSuccess) e = cudaMemcpy(&hs, status, 4, cudaMemcpyDeviceToHost);
+        if (e == cudaSuccess) rc = hs;
+      }
+      if (e != cudaSuccess) cudaGetLastError();
+    }
+  }
+  if (a) cudaFree(a);
+  if (w) cudaFree(w);
+  if (out) cudaFree(out);
+  if (status) cudaFree(status);
+  return rc;
+}
+
 // ---------------------------------------------------------------------------------------------
 // Streaming-read microbenchmark: what a plain read of global memory reaches from a given number of SMs
 // (the HBM denominator for runs on a reduced SM budget).

@@ -72,6 +72,7 @@ struct GemmArgs {
   int plane_w;           // EPI_STORE_PLANES: feature f of token t goes to out[(f / plane_w) * plane_stride + t * plane_w + f % plane_w]
   int64_t plane_stride;  //   (bf16; a K/V cache laid out as planes of [rows][plane_w]); tokens >= n_tok are not stored
   int* status;           // device-visible status word (ADIT_E_TIMEOUT = -6 on an expired wait)
+  int debug_withhold;    // test aid: when n > 0, block 0's token copy of its n-th k-block is never issued (a wait then runs out)
   unsigned long long* dbg;  // optional [grid][16] globaltimer stamps (test aid)
   unsigned long long* trace;  // optional [grid][4]: block start, predecessor-wait released, end, last accumulator complete (%globaltimer ns)
 };
@@ -327,6 +328,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
               ptx::mbar_arrive_expect_tx(&full_bar[stage], w_bytes);
               ptx::tma_load_2d(ws, &map_w, kb * TILE_K, ft * (DUAL ? 2 : 1) * TILE_F, &full_bar[stage]);
             }
+          } else if (g.debug_withhold > 0 && blockIdx.x == 0 && issued + 1 == g.debug_withhold) {
+            // (test aid: this stage never fills; the issuing thread's bounded wait runs out and the block winds down)
           } else {
             ptx::mbar_arrive_expect_tx(&full_bar[stage], a_bytes);
             ptx::tma_load_2d(ws + w_bytes, &map_a, kb * TILE_K, tt * g.tile_tok, &full_bar[stage]);

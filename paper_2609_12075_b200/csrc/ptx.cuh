@@ -51,11 +51,16 @@ __device__ __forceinline__ bool mbar_test_wait(uint64_t* bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
+#ifndef ADIT_WAIT_TRIES
+#define ADIT_WAIT_TRIES 1
+#endif
 // Bounded wait: gives up after `limit_ns` (checked every 1024 polls) and returns false.  The clock read after
 // the first failed test doubles as a short back-off (it takes a few hundred nanoseconds), which measurably
 // helps the warps that share a scheduler with the waiting one.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, uint64_t limit_ns = 2000000000ull) {
-  if (mbar_try_wait(bar, parity)) return true;
+#pragma unroll 1
+  for (int i = 0; i < ADIT_WAIT_TRIES; ++i)
+    if (mbar_try_wait(bar, parity)) return true;
   const uint64_t t0 = globaltimer_ns();
   for (;;) {
 #pragma unroll 1

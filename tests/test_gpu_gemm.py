@@ -70,3 +70,22 @@ def test_budget_does_not_change_a_single_bit(adit):
         outs.append(out.cpu().numpy())
     for o in outs[1:]:
         assert np.array_equal(o.view(np.uint32), outs[0].view(np.uint32))
+
+
+def test_an_expired_wait_ends_the_kernel_with_a_status_and_the_next_launch_is_fine(adit):
+    """Failure detection on the kernel-per-phase path: one block of a small projection is denied one operand copy, its
+    bounded wait runs out (two seconds), the kernel returns by itself with ADIT_E_TIMEOUT in the status word, and the
+    same projection launched again completes with a clean status.  Nothing faults and no wait is unbounded."""
+    import ctypes as C
+    import time
+    import torch
+    first = C.c_int(123)
+    t0 = time.time()
+    rc = adit.lib.adit_debug_gemm_timeout(0, C.byref(first), None)
+    elapsed = time.time() - t0
+    assert first.value == adit.E_TIMEOUT, first.value
+    assert rc == adit.OK, rc
+    assert 1.5 < elapsed < 20.0, elapsed
+    # the device is in working order afterwards
+    x = torch.ones(1024, device="cuda")
+    assert float(x.sum().item()) == 1024.0
