@@ -11,8 +11,8 @@
 //
 // Hand-overs: the ring's "stage filled" barriers live in the even block, which also issues the products; every copy
 // of either block reports its bytes there (the copy's cta_group::2 form lets it name the partner's barrier).  "Stage
-// free" and "accumulator complete" are signalled to both blocks at once by the product pipe (tcgen05.commit to the
-// same barrier offset in both blocks).  "Accumulator drained" is counted in the even block: the odd block's
+// free" and "accumulator complete" are signalled to both blocks by the product pipe (one tcgen05.commit per block, the
+// partner's barrier named by its cluster address).  "Accumulator drained" is counted in the even block: the odd block's
 // epilogue warps arrive remotely.  Every wait is bounded; a block that gave up raises the status word.
 //
 // Warp roles per block (256 threads): warp 0 = weight copies, warp 6 = token copies, warp 1 = tensor-memory

@@ -294,16 +294,17 @@ ADIT_UMMA_KBLOCK2(umma_kblock2_f16_pair, "2")
 // (result wanted one step later), issue this k-block's four products (eight for a gate/up pair), commit them to this
 // stage's "free" barrier, and only then read the test's result - so that the barrier test's latency is hidden behind
 // the products' issue instead of stalling the (in-order) thread.  Returns whether the next stage is already filled.
-// The two-SM form commits to the same barrier offset in both blocks of the pair.  Barriers are given as 32-bit
+// The two-SM form commits to the same barrier offset in both blocks of the pair (two commits: the issuing block's own
+// barrier and, through its cluster address, the partner's - rank 1 of the two-block cluster).  Barriers are given as 32-bit
 // shared-memory addresses (smem_u32), which the caller keeps in registers: every instruction of this thread counts.
 #define ADIT_COMMIT_1 "tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%7];\n\t"
-#define ADIT_COMMIT_2 "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%7], m;\n\t"
+#define ADIT_COMMIT_2 "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%7];\n\tmapa.shared::cluster.u32 pa, %7, 1;\n\ttcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [pa];\n\t"
 #define ADIT_UMMA_STEP(NAME, GROUP, COMMIT)                                                                          \
   __device__ __forceinline__ bool NAME(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t hi, uint32_t idesc,   \
                                        uint32_t acc_first, uint32_t free_bar, uint32_t next_full, uint32_t parity) { \
     uint32_t ready;                                                                                                  \
     asm volatile(                                                                                                    \
-        "{\n\t.reg .pred p, q, r;\n\t.reg .b64 a, b;\n\t.reg .b32 al, bl;\n\t.reg .b16 m;\n\tmov.b16 m, 3;\n\t"     \
+        "{\n\t.reg .pred p, q, r;\n\t.reg .b64 a, b;\n\t.reg .b32 al, bl;\n\t.reg .b32 pa;\n\t"     \
         "mbarrier.test_wait.parity.shared::cta.b64 r, [%8], %9;\n\t"                                                 \
         "setp.ne.b32 p, %6, 0;\n\t"                                                                                  \
         "setp.eq.b32 q, 0, 0;\n\t"                                                                                   \
@@ -328,14 +329,14 @@ ADIT_UMMA_STEP(umma_step_f16_pair, "2", ADIT_COMMIT_2)
 #undef ADIT_COMMIT_1
 #undef ADIT_COMMIT_2
 #define ADIT_COMMIT_1 "tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%9];\n\t"
-#define ADIT_COMMIT_2 "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%9], m;\n\t"
+#define ADIT_COMMIT_2 "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%9];\n\tmapa.shared::cluster.u32 pa, %9, 1;\n\ttcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [pa];\n\t"
 #define ADIT_UMMA_STEP2(NAME, GROUP, COMMIT)                                                                         \
   __device__ __forceinline__ bool NAME(uint32_t d_tmem, uint32_t d_tmem2, uint32_t a_lo, uint32_t a2_lo, uint32_t b_lo, \
                                        uint32_t hi, uint32_t idesc, uint32_t acc_first, uint32_t free_bar,           \
                                        uint32_t next_full, uint32_t parity) {                                       \
     uint32_t ready;                                                                                                  \
     asm volatile(                                                                                                    \
-        "{\n\t.reg .pred p, q, r;\n\t.reg .b64 a, a2, b;\n\t.reg .b32 al, a2l, bl;\n\t.reg .b16 m;\n\tmov.b16 m, 3;\n\t" \
+        "{\n\t.reg .pred p, q, r;\n\t.reg .b64 a, a2, b;\n\t.reg .b32 al, a2l, bl;\n\t.reg .b32 pa;\n\t" \
         "mbarrier.test_wait.parity.shared::cta.b64 r, [%10], %11;\n\t"                                               \
         "setp.ne.b32 p, %8, 0;\n\t"                                                                                  \
         "setp.eq.b32 q, 0, 0;\n\t"                                                                                   \
@@ -428,13 +429,16 @@ __device__ __forceinline__ void umma_f16_pair(uint32_t d_tmem, uint64_t a_desc, 
       "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
-// One arrival on the mbarrier at this shared-memory offset in every block of `cta_mask` (bit = rank in the cluster)
-// once all tcgen05 operations issued so far by this thread are done.
+__device__ __forceinline__ uint32_t mapa_shared(uint32_t local, int rank);
+// One arrival on the mbarrier at this shared-memory offset in the blocks of `cta_mask` (bit 0: the issuing, even block;
+// bit 1: its partner, rank 1 of the two-block cluster) once all tcgen05 operations issued so far by this thread are
+// done: one commit per block, the partner's through its cluster address.
 __device__ __forceinline__ void umma_commit_pair(uint64_t* bar, uint16_t cta_mask) {
-  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(
-                   smem_u32(bar)),
-               "h"(cta_mask)
-               : "memory");
+  const uint32_t local = smem_u32(bar);
+  if (cta_mask & 1)
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(local) : "memory");
+  if (cta_mask & 2)
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(mapa_shared(local, 1)) : "memory");
 }
 // 2-D tiled load into this block's shared memory whose completion is counted on an mbarrier that may live in the
 // other block of the pair (`bar_cluster` is a shared::cluster address, see mapa_shared).
