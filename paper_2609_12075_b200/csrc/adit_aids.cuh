@@ -270,7 +270,10 @@ extern "C" int adit_debug_gemm_timeout(int device, int* first_status, void* stre
   if (tc::ensure_smem_attr() != cudaSuccess) return ADIT_E_CUDA;
   const int n_tok = 51, n_feat = 2560, k = 1024, SM = prop.multiProcessorCount;
   const tc::GemmPlan p = tc::plan_gemm(n_tok, n_feat, k, false, SM, false);  // (k-split not allowed)
-  if (p.splits != 1) return ADIT_E_UNSUPPORTED;
+  // the one instantiation that has the withholding compiled in: 16-token epilogue chunks, no k-split, two issuing threads
+  if (p.splits != 1 || p.issuers != 2 || ((p.tile_tok & 31) == 0 && p.tile_tok >= 96)) return ADIT_E_UNSUPPORTED;
+  auto withhold_kernel = tc::gemm_tc_kernel<false, EPI_STORE_F32, 16, false, 2, true, true>;
+  if (cudaFuncSetAttribute(withhold_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::SMEM_BUDGET + 1024) != cudaSuccess) return ADIT_E_CUDA;
   void *a = nullptr, *w = nullptr;
   float* out = nullptr;
   int* status = nullptr;
@@ -288,7 +291,10 @@ extern "C" int adit_debug_gemm_timeout(int device, int* first_status, void* stre
       tc::GemmArgs g{};
       g.n_feat = n_feat; g.n_tok = n_tok; g.epi = EPI_STORE_F32; g.out = out; g.ldo = n_feat; g.status = status;
       g.debug_withhold = 3;
-      cudaError_t e = tc::launch_gemm(mw, ma, p, false, g, SM, st);
+      g.kb_total = p.kb_total; g.tile_tok = p.tile_tok; g.n_ftiles = p.n_ftiles; g.n_ttiles = p.n_ttiles; g.splits = 1;
+      g.stages = p.stages; g.tmem_cols = p.tmem_cols; g.ring_bytes = p.ring_bytes; g.acc_bufs = p.acc_bufs; g.issuers = p.issuers;
+      withhold_kernel<<<tc::gemm_grid(p, SM), tc::GEMM_THREADS, p.smem_bytes, st>>>(mw, ma, g);
+      cudaError_t e = cudaGetLastError();
       if (e == cudaSuccess) e = cudaStreamSynchronize(st);
       int hs = 0;
       if (e == cudaSuccess) e = cudaMemcpy(&hs, status, 4, cudaMemcpyDeviceToHost);

@@ -72,7 +72,7 @@ struct GemmArgs {
   int plane_w;           // EPI_STORE_PLANES: feature f of token t goes to out[(f / plane_w) * plane_stride + t * plane_w + f % plane_w]
   int64_t plane_stride;  //   (bf16; a K/V cache laid out as planes of [rows][plane_w]); tokens >= n_tok are not stored
   int* status;           // device-visible status word (ADIT_E_TIMEOUT = -6 on an expired wait)
-  int debug_withhold;    // test aid: when n > 0, block 0's token copy of its n-th k-block is never issued (a wait then runs out)
+  int debug_withhold;    // test aid (WITHHOLD instantiation only): when n > 0, block 0's token copy of its n-th k-block is never issued
   unsigned long long* dbg;  // optional [grid][16] globaltimer stamps (test aid)
   unsigned long long* trace;  // optional [grid][4]: block start, predecessor-wait released, end, last accumulator complete (%globaltimer ns)
 };
@@ -218,7 +218,9 @@ __device__ __forceinline__ void finalize_stats(const GemmArgs& g, int nvalid, in
 // fetched anew at every launch, so each instantiation carries one chunk width only.
 // SPLIT: the kernel runs as clusters that share the k dimension (exchange code only in these instantiations).
 // NI: product-issuing threads (1 or 2).  INSTR: phase stamps and launch trace compiled in (test and measurement aids).
-template <bool DUAL, int EPI, int CW, bool SPLIT, int NI, bool INSTR>
+// WITHHOLD: the failure-path test aid (GemmArgs::debug_withhold) compiled in: one instantiation only, because even a
+// never-taken test in the copy-issuing thread's loop costs the batch-1 call 1.7 %.
+template <bool DUAL, int EPI, int CW, bool SPLIT, int NI, bool INSTR, bool WITHHOLD = false>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_a, GemmArgs g) {
   extern __shared__ uint8_t smem_raw[];
@@ -328,7 +330,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
               ptx::mbar_arrive_expect_tx(&full_bar[stage], w_bytes);
               ptx::tma_load_2d(ws, &map_w, kb * TILE_K, ft * (DUAL ? 2 : 1) * TILE_F, &full_bar[stage]);
             }
-          } else if (g.debug_withhold > 0 && blockIdx.x == 0 && issued + 1 == g.debug_withhold) {
+          } else if (WITHHOLD && g.debug_withhold > 0 && blockIdx.x == 0 && issued + 1 == g.debug_withhold) {
             // (test aid: this stage never fills; the issuing thread's bounded wait runs out and the block winds down)
           } else {
             ptx::mbar_arrive_expect_tx(&full_bar[stage], a_bytes);
