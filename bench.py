@@ -683,14 +683,18 @@ def run_lockstep(args):
     eng.load_weights(W.make_weights(cfg, wl.seed))
     inputs = {"pi0": {"kv": adit.upload_prefix_kv(wl), "len": wl.prefix_len, "state": torch.from_numpy(wl.state).cuda(),
                       "noise": torch.from_numpy(wl.noise).cuda(), "steps": wl.n_steps}}
-    stages = LS.GpuStages(adit, {"pi0": eng}, inputs, vlm_iters_per_request=args.vlm_iters)
+    stages = LS.GpuStages(adit, {"pi0": eng}, inputs, vlm_iters_per_request=args.vlm_iters, restriction="green" if args.green else "grid")
     for b in LS.batch_sizes(max_batch):               # record every batch size's launch graph first
         stages.time_lockstep("pi0", b, b, 0, reps=1)
     t0 = time.perf_counter()
-    table = LS.SmTable.profile(stages.n_sm, max_batch, lambda vb, ab, cap: stages.time_lockstep("pi0", vb, ab, cap, reps=2))
+    # the paper's arrangement: only the VLM stream is restricted, the ADiT call runs unrestricted
+    table = LS.SmTable.profile(stages.n_sm, max_batch, lambda vb, ab, cap: stages.time_lockstep("pi0", vb, ab, cap, reps=2, arrangement="vlm_only"),
+                               arrangement="vlm_only")
+    # both stages with an explicit allotment (the ADiT call's sm_budget = the SMs outside the VLM's)
+    table_c = LS.SmTable.profile(stages.n_sm, max_batch, lambda vb, ab, cap: stages.time_lockstep("pi0", vb, ab, cap, reps=2))
     profile_s = time.perf_counter() - t0
     out = {}
-    for name, tab in (("guarded", table), ("unguarded", LS.SmTable(stages.n_sm))):
+    for name, tab in (("guarded", table), ("guarded_complement", table_c), ("unguarded", LS.SmTable(stages.n_sm))):
         ex = LS.LockstepExecutor(stages.vlm, stages.adit_stage, max_batch, tab, {"pi0": 156_000})
         reqs = [LS.Request("pi0", i, 0, payload=i % pool) for i in range(args.requests)]
         [ex.submit(r) for r in reqs]
@@ -705,11 +709,16 @@ def run_lockstep(args):
     assert eng.poll_status() == 0
     print(json.dumps({"metric": "lockstep_time_with_profiled_sm_restriction", "unit": "ms", "config": {
         "expert": "pi0-scale, 816-token prefixes, 10 Euler steps", "max_batch": max_batch,
-        "vlm_stand_in": f"bf16 GEMM 8192x2048x2048 x {args.vlm_iters} per request, grid capped to the restriction",
+        "vlm_stand_in": f"bf16 GEMM 8192x2048x2048 x {args.vlm_iters} per request, " +
+                        ("full grid on a green-context stream of the restriction's SMs" if args.green else "grid capped to the restriction"),
+        "arrangements": "guarded = only the VLM stream restricted (the paper's); guarded_complement = the ADiT call's sm_budget is the rest",
         "candidates": "multiples of 8 SMs and no restriction", "n_sm": stages.n_sm, "profile_seconds": profile_s},
         "table": {f"{vb},{ab}": c for (vb, ab), c in sorted(table.entries.items())},
         "table_ms": {f"{vb},{ab}": {"best": 1e3 * t[table.entries[(vb, ab)]], "unrestricted": 1e3 * t[0]}
                      for (vb, ab), t in sorted(table.times.items())},
+        "table_complement": {f"{vb},{ab}": c for (vb, ab), c in sorted(table_c.entries.items())},
+        "table_complement_ms": {f"{vb},{ab}": {"best": 1e3 * t[table_c.entries[(vb, ab)]], "unrestricted": 1e3 * t[0]}
+                                for (vb, ab), t in sorted(table_c.times.items())},
         "trace": out, "speedup_guarded_vs_unguarded": out["unguarded"]["total_s"] / out["guarded"]["total_s"]}))
     stages.close()
     eng.close()
@@ -734,7 +743,7 @@ def main():
     ap.add_argument("--no-trace", action="store_true", help="skip the in-situ timeline of one call")
     ap.add_argument("--no-extra", action="store_true", help="skip the brief runs of the other batch sizes (c3, c4)")
     ap.add_argument("--no-graph", action="store_true", help="enqueue kernels one by one (ADIT_FLAG_NO_GRAPH): for profilers")
-    ap.add_argument("--green", action="store_true", help="sweep: also run the load on a green-context stream confined to the SMs outside the budget, the call unrestricted")
+    ap.add_argument("--green", action="store_true", help="sweep: also run the load on a green-context stream confined to the SMs outside the budget, the call unrestricted; lockstep: restrict the VLM stand-in with green-context streams instead of grid caps")
     ap.add_argument("--one-sm-gemm", action="store_true", help="projections on the one-SM kernel at every batch size (ADIT_FLAG_ONE_SM_GEMM): comparison")
     ap.add_argument("--persistent", action="store_true", help="small batches as one persistent kernel (ADIT_FLAG_PERSISTENT_LOOP)")
     ap.add_argument("--latency-calls", type=int, default=None, help="calls sampled for p50/p99 (default 1000 at batch 1)")

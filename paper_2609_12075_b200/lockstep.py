@@ -55,7 +55,12 @@ class SmTable:
     """(VLM batch size, ADiT batch size) -> SMs the VLM stream is restricted to (0: no restriction)."""
 
     def __init__(self, n_sm: int, entries: Optional[Dict[Tuple[int, int], int]] = None,
-                 times: Optional[Dict[Tuple[int, int], Dict[int, float]]] = None):
+                 times: Optional[Dict[Tuple[int, int], Dict[int, float]]] = None, arrangement: str = "complement"):
+        # arrangement: what the ADiT call gets beside a restricted VLM stream - "complement": an sm_budget of the
+        # remaining SMs (both stages take an explicit allotment); "vlm_only": no restriction (the paper's arrangement:
+        # only the VLM stream is confined, the ADiT kernels run wherever SMs are free)
+        assert arrangement in ("complement", "vlm_only")
+        self.arrangement = arrangement
         self.n_sm = int(n_sm)
         self.entries: Dict[Tuple[int, int], int] = dict(entries or {})
         self.times: Dict[Tuple[int, int], Dict[int, float]] = dict(times or {})
@@ -67,16 +72,18 @@ class SmTable:
     def budgets(self, vlm_batch: int, adit_batch: int) -> Tuple[int, int]:
         """(SMs for the VLM stream, sm_budget of the ADiT call); (0, 0) = both unrestricted."""
         cap = self.lookup(vlm_batch, adit_batch)
-        return (cap, self.n_sm - cap) if cap > 0 else (0, 0)
+        if cap <= 0:
+            return (0, 0)
+        return (cap, self.n_sm - cap) if self.arrangement == "complement" else (cap, 0)
 
     @classmethod
     def profile(cls, n_sm: int, max_batch: int, time_lockstep: Callable[[int, int, int], float], step: int = 8,
-                candidates: Optional[Sequence[int]] = None) -> "SmTable":
+                candidates: Optional[Sequence[int]] = None, arrangement: str = "complement") -> "SmTable":
         """Offline sweep: for every pair of batch sizes time a lockstep under every candidate restriction
         (`time_lockstep(vlm_batch, adit_batch, vlm_sms)` returns seconds; vlm_sms = 0 means unrestricted) and keep the
         fastest.  Ties go to the smaller restriction index, i.e. to the candidate tried first."""
         cand = list(candidates) if candidates is not None else sm_candidates(n_sm, step)
-        table = cls(n_sm)
+        table = cls(n_sm, arrangement=arrangement)
         for vb in batch_sizes(max_batch):
             for ab in batch_sizes(max_batch):
                 t = {c: float(time_lockstep(vb, ab, c)) for c in cand}
@@ -86,7 +93,7 @@ class SmTable:
         return table
 
     def to_json(self) -> str:
-        return json.dumps({"n_sm": self.n_sm,
+        return json.dumps({"n_sm": self.n_sm, "arrangement": self.arrangement,
                            "entries": [[vb, ab, c] for (vb, ab), c in sorted(self.entries.items())],
                            "times": [[vb, ab, {str(c): v for c, v in t.items()}] for (vb, ab), t in sorted(self.times.items())]})
 
@@ -94,7 +101,8 @@ class SmTable:
     def from_json(cls, text: str) -> "SmTable":
         d = json.loads(text)
         return cls(d["n_sm"], {(vb, ab): c for vb, ab, c in d["entries"]},
-                   {(vb, ab): {int(c): v for c, v in t.items()} for vb, ab, t in d.get("times", [])})
+                   {(vb, ab): {int(c): v for c, v in t.items()} for vb, ab, t in d.get("times", [])},
+                   arrangement=d.get("arrangement", "complement"))
 
 
 @dataclass
@@ -225,8 +233,13 @@ class GpuStages:
     adit_denoise as the ADiT stage, each on its own stream and synchronised by its own thread."""
 
     def __init__(self, adit_mod, engines: Dict[str, object], inputs: Dict[str, dict], vlm_iters_per_request: int = 6,
-                 gemm_shape: Tuple[int, int, int] = (8192, 2048, 2048), device: int = 0):
+                 gemm_shape: Tuple[int, int, int] = (8192, 2048, 2048), device: int = 0, restriction: str = "grid"):
+        # restriction: how the VLM stream is held to its SMs - "grid": the stand-in's grid is capped (it honours a cap);
+        # "green": its full grid runs on a green-context stream of that many SMs (the paper's mechanism, which also
+        # confines kernels that were not written for a budget)
         import torch
+        assert restriction in ("grid", "green")
+        self.restriction, self.device, self._green = restriction, device, {}
         self.torch, self.adit = torch, adit_mod
         self.engines, self.inputs = engines, inputs
         self.vlm_iters = int(vlm_iters_per_request)
@@ -235,10 +248,15 @@ class GpuStages:
         self.n_sm = torch.cuda.get_device_properties(device).multi_processor_count
 
     def vlm(self, model: str, requests: List[Request], sms: int):
-        self.bg.launch(self.vlm_iters * len(requests), sms, self.s_vlm)
+        stream = self.s_vlm
+        if self.restriction == "green" and sms > 0:
+            if sms not in self._green:
+                self._green[sms] = self.adit.GreenStream(sms, device=self.device)
+            stream, sms = self._green[sms].stream, 0     # the driver confines the full grid
+        self.bg.launch(self.vlm_iters * len(requests), sms, stream)
         for r in requests:                              # hand-over: the request's (precomputed) prefix cache
             r.vlm_output = r.payload
-        self.s_vlm.synchronize()
+        stream.synchronize()
 
     def adit_stage(self, model: str, requests: List[Request], sms: int):
         torch = self.torch
@@ -251,14 +269,15 @@ class GpuStages:
         for j, r in enumerate(requests):
             r.result = out[j]
 
-    def time_lockstep(self, model: str, vlm_batch: int, adit_batch: int, vlm_sms: int, reps: int = 3) -> float:
+    def time_lockstep(self, model: str, vlm_batch: int, adit_batch: int, vlm_sms: int, reps: int = 3,
+                      arrangement: str = "complement") -> float:
         """Seconds for one lockstep of this pair (both stages launched together, until both are done), best of reps."""
         best = float("inf")
         reqs_v = [Request(model, i, 0, payload=i % len(self.inputs[model]["kv"])) for i in range(vlm_batch)]
         reqs_a = [Request(model, i, 0, payload=i % len(self.inputs[model]["kv"])) for i in range(adit_batch)]
         for r in reqs_a:
             r.vlm_output = r.payload
-        adit_sms = self.n_sm - vlm_sms if vlm_sms > 0 else 0
+        adit_sms = self.n_sm - vlm_sms if (vlm_sms > 0 and arrangement == "complement") else 0
         for _ in range(reps + 1):
             self.torch.cuda.synchronize()
             t0 = time.perf_counter()
@@ -269,4 +288,7 @@ class GpuStages:
         return best
 
     def close(self):
+        for g in self._green.values():
+            g.close()
+        self._green = {}
         self.bg.close()

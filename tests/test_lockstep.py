@@ -37,6 +37,10 @@ def test_profile_keeps_the_fastest_restriction_per_batch_pair():
     # light ADiT batch: giving up an eighth of the chip costs more than running the ADiT stage afterwards
     assert table.lookup(1, 4) == 56 and table.lookup(4, 1) == 0
     assert table.budgets(1, 4) == (56, 8) and table.budgets(8, 8) == (0, 0)      # unprofiled pair: unrestricted
+    # the paper's arrangement: only the VLM stream is restricted, the ADiT call gets no budget (0 = unrestricted)
+    paper = L.SmTable.profile(n_sm, 4, t, arrangement="vlm_only")
+    assert paper.entries == table.entries and paper.budgets(1, 4) == (56, 0) and paper.budgets(4, 1) == (0, 0)
+    assert L.SmTable.from_json(paper.to_json()).arrangement == "vlm_only" and L.SmTable.from_json(table.to_json()).arrangement == "complement"
     back = L.SmTable.from_json(table.to_json())
     assert back.entries == table.entries and back.n_sm == n_sm and back.times[(2, 1)][56] == t(2, 1, 56) and back.lookup(1, 4) == 56
     # when restricting never pays, the table says "no restriction"
