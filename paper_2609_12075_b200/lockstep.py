@@ -10,8 +10,9 @@ O(log max_batch) batch sizes occur - and the number of SMs the VLM stream may us
 pair under every restriction in multiples of 8 SMs, and under no restriction, and keeps the fastest.
 
 In the paper the restriction is applied to the VLM stream (Green Contexts) and the ADiT kernels find the remaining
-SMs free.  Here both stages take an explicit SM allotment - the VLM stand-in is a GEMM loop whose grid is capped, the
-ADiT call gets sm_budget = the rest - and "no restriction" means both may use the whole chip.
+SMs free: the table's arrangement "vlm_only".  The arrangement "complement" gives both stages an explicit SM
+allotment instead - the ADiT call gets sm_budget = the rest.  "No restriction" means both may use the whole chip.
+The VLM stand-in is a GEMM loop; its restriction is a cap on its grid or, as in the paper, a green-context stream.
 
 The executor is host code and independent of CUDA: a stage is any callable that runs a batch to completion on its
 own stream.  `GpuStages` supplies the two callables used on a B200.
