@@ -114,6 +114,16 @@ def test_hand_over_errors(adit):
         eng.load_prefix_projection(bad)
     assert e.value.code == adit.E_INVALID
     eng.load_prefix_projection(pw)
+    # (the smallest shape family, head_dim 64 and a hidden width of one k-block, also projects correctly)
+    hid = [W.make_prefix_hidden(3, b, p, 64) for b, p in enumerate((32, 7))]
+    small = _empty_caches(cfg, 2, 32)
+    eng.project_prefix([torch.from_numpy(x).to(torch.bfloat16).cuda() for x in hid], [32, 7], small)
+    torch.cuda.synchronize()
+    for b, P in enumerate((32, 7)):
+        got = small[b].float().cpu().numpy().astype(np.float64)
+        ref = O.project_prefix_kv(cfg, hid[b], pw, 32, pad_value=-3.0)
+        assert np.all(got[:, :, :, P:, :] == -3.0)
+        assert np.all(np.abs(got[:, :, :, :P] - ref[:, :, :, :P]) <= 2.0 ** -8 * np.abs(ref[:, :, :, :P]) + 1e-3)
     caches = _empty_caches(cfg, 3, 32)
     h = [torch.zeros(8, 64, dtype=torch.bfloat16, device="cuda") for _ in range(3)]
     with pytest.raises(adit.AditError) as e:
