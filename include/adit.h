@@ -380,6 +380,15 @@ int adit_debug_stamps_selected(int armed_device, int device, int grid_blocks, in
 int adit_debug_plan(int n_tok, int n_feat, int k, int dual, int sm_count, int32_t* out);
 
 /*
+ * adit_debug_plan_projection: as adit_debug_plan, but the plan a projection of the loop actually runs with: when
+ * `allow_pair` is non-zero (the default of the loop; ADIT_FLAG_ONE_SM_GEMM clears it) large gate/up pairs go to
+ * the kernel that runs one tile on a pair of SMs.  Writes thirteen int32: the twelve of adit_debug_plan, then 1 if
+ * the two-SM kernel was chosen (the tile then spans 256 features on two blocks, each of which brings in half of the
+ * token tile), else 0.  Host-only; returns ADIT_OK or ADIT_E_INVALID.
+ */
+int adit_debug_plan_projection(int n_tok, int n_feat, int k, int dual, int sm_count, int allow_pair, int32_t* out);
+
+/*
  * adit_debug_stream_read: measurement aid (no counterpart in the paper).  Allocates `bytes` of device memory
  * (larger than the L2 cache to measure HBM), reads it `iters` times with one thread block of 512 threads on each
  * of `sm_count` SMs using 16-byte loads, and writes the achieved read bandwidth in GB/s: the memory roofline

@@ -27,7 +27,7 @@ MAX_BATCH, MAX_STEPS = 64, 64
 
 EXPORTS = ["adit_create", "adit_load_weights", "adit_denoise", "adit_denoise_host", "adit_destroy",
            "adit_poll_status", "adit_last_cuda_error", "adit_kernel_launches", "adit_strerror",
-           "adit_debug_copy", "adit_debug_gemm", "adit_debug_gemm_timeout", "adit_debug_plan", "adit_debug_gemm_stamps", "adit_debug_attention", "adit_attention_static", "adit_profile_enable", "adit_profile_read", "adit_profile_class_name", "adit_trace_enable", "adit_trace_read",
+           "adit_debug_copy", "adit_debug_gemm", "adit_debug_gemm_timeout", "adit_debug_plan", "adit_debug_plan_projection", "adit_debug_gemm_stamps", "adit_debug_attention", "adit_attention_static", "adit_profile_enable", "adit_profile_read", "adit_profile_class_name", "adit_trace_enable", "adit_trace_read",
            "adit_load_prefix_projection", "adit_project_prefix", "adit_green_stream_create", "adit_green_stream_handle", "adit_green_stream_sm_count", "adit_green_stream_destroy", "adit_bg_gemm_create", "adit_bg_gemm_create_kind", "adit_bg_gemm_launch", "adit_bg_gemm_destroy",
            "adit_debug_stream_read", "adit_attention_static_status", "adit_debug_stamps_selected",
            "adit_clear_status", "adit_uses_persistent_loop", "adit_debug_wait_limit", "adit_loop_trace_read"]
@@ -66,6 +66,8 @@ N_KERNEL_CLASSES = 11
 lib.adit_debug_gemm_stamps.argtypes = [C.c_void_p, C.c_int]
 lib.adit_debug_plan.argtypes = [C.c_int] * 5 + [C.POINTER(C.c_int32)]
 lib.adit_debug_plan.restype = C.c_int
+lib.adit_debug_plan_projection.argtypes = [C.c_int] * 6 + [C.POINTER(C.c_int32)]
+lib.adit_debug_plan_projection.restype = C.c_int
 lib.adit_debug_gemm_timeout.argtypes = [C.c_int, C.POINTER(C.c_int), C.c_void_p]
 lib.adit_debug_gemm.argtypes = [C.c_int, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int,
                                 C.c_void_p]
@@ -283,6 +285,18 @@ def debug_plan(n_tok: int, n_feat: int, k: int, dual: bool = False, sm_count: in
         raise AditError(rc)
     names = ("tile_tok", "n_ttiles", "n_ftiles", "splits", "stages", "kb_total", "acc_bufs", "issuers", "tmem_cols",
              "smem_bytes", "ring_bytes", "est_ns")
+    return dict(zip(names, out))
+
+
+def debug_plan_projection(n_tok: int, n_feat: int, k: int, dual: bool = False, sm_count: int = 148,
+                          allow_pair: bool = True) -> dict:
+    """The plan a projection of the loop runs with, `pair` = 1 where it is the two-SM kernel (host-only)."""
+    out = (C.c_int32 * 13)()
+    rc = lib.adit_debug_plan_projection(n_tok, n_feat, k, int(dual), sm_count, int(allow_pair), out)
+    if rc != 0:
+        raise AditError(rc)
+    names = ("tile_tok", "n_ttiles", "n_ftiles", "splits", "stages", "kb_total", "acc_bufs", "issuers", "tmem_cols",
+             "smem_bytes", "ring_bytes", "est_ns", "pair")
     return dict(zip(names, out))
 
 

@@ -196,6 +196,15 @@ extern "C" int adit_debug_plan(int n_tok, int n_feat, int k, int dual, int sm_co
   return ADIT_OK;
 }
 
+extern "C" int adit_debug_plan_projection(int n_tok, int n_feat, int k, int dual, int sm_count, int allow_pair, int32_t* out) {
+  if (!out || n_tok < 1 || n_feat < 1 || k < 64 || (k % 64) || sm_count < 1) return ADIT_E_INVALID;
+  const tc::GemmPlan p = tc::plan_projection(n_tok, n_feat, k, dual != 0, sm_count, allow_pair != 0);
+  out[0] = p.tile_tok; out[1] = p.n_ttiles; out[2] = p.n_ftiles; out[3] = p.splits; out[4] = p.stages; out[5] = p.kb_total;
+  out[6] = p.acc_bufs; out[7] = p.issuers; out[8] = (int32_t)p.tmem_cols; out[9] = (int32_t)p.smem_bytes;
+  out[10] = (int32_t)p.ring_bytes; out[11] = (int32_t)(p.est_us * 1000.0); out[12] = p.pair ? 1 : 0;
+  return ADIT_OK;
+}
+
 extern "C" int adit_debug_gemm_stamps(unsigned long long* host_dst, int n_blocks) {
   if (!host_dst && n_blocks < 0) {  // disarm
     if (g_gemm_dbg) { cudaSetDevice(g_gemm_dbg_device); cudaDeviceSynchronize(); cudaFree(g_gemm_dbg); }

@@ -49,3 +49,24 @@ def test_plan_is_deterministic_and_rejects_bad_arguments():
     for bad in ((0, 128, 64), (16, 0, 64), (16, 128, 0), (16, 128, 100)):
         with pytest.raises(adit.AditError):
             adit.debug_plan(*bad)
+
+
+@pytest.mark.parametrize("sm_count", [148, 132, 16, 2])
+def test_projection_plan_uses_the_two_sm_kernel_only_where_it_may(sm_count):
+    for n_tok, n_feat, k, dual in SHAPES + [(n, 4096, 1024, True) for n in (1023, 1024, 1025, 2000, 8192)]:
+        one = adit.debug_plan(n_tok, n_feat, k, dual, sm_count)
+        off = adit.debug_plan_projection(n_tok, n_feat, k, dual, sm_count, allow_pair=False)
+        assert off.pop("pair") == 0 and off == one                              # the flag that forbids it gives the one-SM plan
+        p = adit.debug_plan_projection(n_tok, n_feat, k, dual, sm_count)
+        what = (n_tok, n_feat, k, dual, sm_count, p)
+        if not (dual and n_tok >= 1024 and k >= 128):
+            assert p.pop("pair") == 0 and p == one, what
+            continue
+        assert p["pair"] == 1 and p["splits"] == 1 and p["issuers"] == 1, what
+        assert p["tile_tok"] % 16 == 0 and 32 <= p["tile_tok"] <= 256, what     # each block brings in half: whole 8-row groups
+        assert p["n_ttiles"] * p["tile_tok"] >= n_tok, what
+        assert p["n_ttiles"] * p["tile_tok"] - n_tok < 320, what
+        assert p["acc_bufs"] in (1, 2) and p["acc_bufs"] * 2 * p["tile_tok"] <= p["tmem_cols"] <= 512, what
+        stage = 2 * 128 * 64 * 2 + (p["tile_tok"] // 2) * 64 * 2                # this block's weight rows + its half of the tokens
+        assert 2 <= p["stages"] <= 12 and p["ring_bytes"] == p["stages"] * stage, what
+        assert p["smem_bytes"] == p["ring_bytes"] + 1024 <= 217 * 1024, what
