@@ -212,6 +212,32 @@ def step_roofline(cfg, prefix_len, n_euler, ms_per_call, peaks):
                   "achieved_tflops": work["step_flops"] * n_euler / (ms_per_call * 1e-3) / 1e12}
 
 
+def layer_timeline(trace, names):
+    """Per kernel class, medians in microseconds over the traced launches of: `interval` = this kernel's dependency
+    release to the next kernel's (what the kernel adds to the call), `main` = release to the last accumulator complete,
+    `epilogue` = from there to the last block's end, `handover` = the rest of the interval.  Rows of `trace`: class,
+    blocks, first/last block start, first/last block end, first/last release, first/last accumulator complete (ns;
+    0 where a kernel has no such stamp)."""
+    out = {}
+    for c in sorted(set(int(x) for x in trace[:-1, 0])):
+        idx = np.where(trace[:-1, 0] == c)[0]
+        m, nxt = trace[idx], trace[idx + 1]
+        ok = (m[:, 7] > 0) & (nxt[:, 7] > 0)
+        if not ok.any():
+            continue
+        m, nxt = m[ok], nxt[ok]
+        row = {"launches": int(len(m)), "blocks": int(np.median(m[:, 1])), "interval": float(np.median(nxt[:, 7] - m[:, 7])) / 1e3}
+        has_main = m[:, 9] > 0
+        if has_main.all():
+            row["main"] = float(np.median(m[:, 9] - m[:, 7])) / 1e3
+            row["epilogue"] = float(np.median(m[:, 5] - m[:, 9])) / 1e3
+            row["handover"] = row["interval"] - row["main"] - row["epilogue"]
+        else:
+            row["release_to_end"] = float(np.median(m[:, 5] - m[:, 7])) / 1e3
+        out[names[c]] = row
+    return out
+
+
 def sample_latency(torch, eng, sets, n_euler, budget, stream, n_calls, wall_s):
     """Per-call device latency (CUDA events on the call's stream) of up to n_calls back-to-back calls, stopped early
     when the wall budget is spent."""
@@ -396,6 +422,12 @@ def run_ours(args):
                     "serialised_events": serialised,
                     "peak_source": f"{peaks_kind} (MEASURED_PEAKS.json)" if peaks_kind == "measured" else "fallback"}
 
+    # ---- where a call's time goes: per kernel class, from the same in-situ stamps (medians over the traced launches) ----
+    timeline = None
+    if trace is not None and len(trace) > 1:
+        timeline = layer_timeline(np.asarray(trace, dtype=np.int64),
+                                  [adit.lib.adit_profile_class_name(i).decode() for i in range(adit.N_KERNEL_CLASSES)])
+
     # ---- the other batch sizes of the metric, briefly (same expert, its own handle sized for 32 requests) ----
     by_workload = {}
     if world == 1 and args.workload == "c2" and not args.no_extra:
@@ -473,7 +505,7 @@ def run_ours(args):
         "config": bench_config(base, args.sm_budget, world, work["step_bytes"], n_sets),
         "latency_ms": {"p50": float(np.percentile(lat, 50)), "p99": float(np.percentile(lat, 99)),
                        "mean": float(lat.mean()), "min": float(lat.min()), "calls": int(len(lat))},
-        "roofline": roofline, "roofline_step": step_roof, "kernel_shares": shares, "by_workload": by_workload,
+        "roofline": roofline, "roofline_step": step_roof, "kernel_shares": shares, "timeline_us": timeline, "by_workload": by_workload,
         "cpu_baseline": cpu,
         "e2e": {"value": world * B * n_e2e / e2e_s, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "calls": n_e2e},

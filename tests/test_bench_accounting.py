@@ -46,3 +46,17 @@ def test_traffic_is_read_from_the_committed_profile_summaries():
     assert t is not None and 8.0e6 < t < 1.0e7         # measured DRAM bytes of one projection launch (8.65 MB algorithmic)
     assert bench.traffic_from_profile("no_such_kernel", "c2") is None
     assert os.path.exists(os.path.join(bench.ROOT, "profiles", "gemm_tc_kernel_c2.md"))
+
+
+def test_layer_timeline_on_a_synthetic_trace():
+    import numpy as np
+    rows, t = [], 1000
+    for i in range(6):  # two kernel classes in turn, 5 us apart; only class 0 stamps its accumulators
+        c = i % 2
+        rows.append([c, 64, t - 500, t - 400, t + 3000, t + 3500, t, t + 10, t + 2000 if c == 0 else 0, t + 2500 if c == 0 else 0])
+        t += 5000
+    tl = bench.layer_timeline(np.array(rows, dtype=np.int64), ["a", "b"])
+    a, b = tl["a"], tl["b"]
+    assert a["launches"] == 3 and a["blocks"] == 64 and a["interval"] == 5.0
+    assert abs(a["main"] - 2.49) < 1e-9 and abs(a["epilogue"] - 1.0) < 1e-9 and abs(a["handover"] - 1.51) < 1e-9
+    assert b["launches"] == 2 and abs(b["release_to_end"] - 3.49) < 1e-9 and "main" not in b   # (the last launch has no successor)
