@@ -296,7 +296,9 @@ int adit_debug_gemm_timeout(int device, int* first_status, void* stream);
 /*
  * adit_debug_gemm: run the tensor-core projection kernel on its own (test aid): out[n_tok, n_feat]
  * (fp32, device) = A[n_tok, k] W[n_feat, k]^T with bf16 device operands, k a multiple of 64;
- * splits = 0 lets the library choose the k-split, splits = -2 selects the two-SM kernel (pairs of
+ * splits = 0 lets the library choose the k-split, 1..8 caps it, 100 * t + c (t >= 1) additionally fixes the
+ * number of token tiles at t (for sweeps of the tiling; a combination the kernel has no room for falls back to
+ * the nearest admissible one), splits = -2 selects the two-SM kernel (pairs of
  * thread blocks, 256 features x tile_tokens per pair), sm_budget as in adit_denoise.  Synchronises the
  * stream.  Returns a negative status, or a positive plan code splits * 1e6 + tile_tokens * 1e3 +
  * pipeline stages (splits reads 9 for the two-SM kernel).  The paper has no counterpart.

@@ -234,7 +234,7 @@ extern "C" int adit_debug_gemm(int device, int n_tok, int n_feat, int k, const v
   if (tc::ensure_smem_attr() != cudaSuccess) return ADIT_E_CUDA;
   const int SM = prop.multiProcessorCount;
   if (splits == -2 && SM < 2) return ADIT_E_UNSUPPORTED;
-  tc::GemmPlan p = splits == -2 ? tc::plan_gemm_pair(n_tok, n_feat, k, false, SM) : tc::plan_gemm(n_tok, n_feat, k, false, SM, true, splits);
+  tc::GemmPlan p = splits == -2 ? tc::plan_gemm_pair(n_tok, n_feat, k, false, SM) : tc::plan_gemm(n_tok, n_feat, k, false, SM, true, splits % 100, splits / 100);
   CUtensorMap mw, ma;
   if (!tc::make_map_bf16(&mw, w_bf16, n_feat, k, tc::TILE_F) || !tc::make_map_bf16(&ma, a_bf16, n_tok, k, tc::token_box_rows(p)))
     return ADIT_E_CUDA;

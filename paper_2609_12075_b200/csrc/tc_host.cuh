@@ -76,7 +76,8 @@ struct GemmPlan {
 // costs about 0.5 us per 32 tokens (only the last tile's is exposed); and a k-split over a cluster adds
 // parking the accumulator, the exchange through distributed shared memory (about 20 GB/s into each
 // block), the rank-order sum and a cluster barrier.
-static GemmPlan plan_gemm(int n_tok, int n_feat, int K, bool dual, int sm_count, bool allow_split, int force_splits = 0) {
+static GemmPlan plan_gemm(int n_tok, int n_feat, int K, bool dual, int sm_count, bool allow_split, int force_splits = 0,
+                          int force_ttiles = 0) {
   GemmPlan p;
   const int nv = dual ? 2 : 1;
   p.n_ftiles = (n_feat + TILE_F - 1) / TILE_F;
@@ -88,6 +89,7 @@ static GemmPlan plan_gemm(int n_tok, int n_feat, int K, bool dual, int sm_count,
     const int tile16 = (((n_tok + nt - 1) / nt) + 15) / 16 * 16;
     if (tile16 > 256) continue;
     if (nt > 1 && tile16 < 32) break;
+    if (force_ttiles > 0 && nt != force_ttiles) continue;  // test aid
     for (int cs = 8; cs >= 1; cs >>= 1) {
       if (cs > 1 && !allow_split && force_splits <= 0) continue;
       if (force_splits > 0 && cs > force_splits) continue;
