@@ -70,7 +70,9 @@ struct GemmPlan {
 // the same for any budget.
 //
 // The choice minimises an estimate of the kernel's duration built from figures measured on B200 with this
-// kernel: a k-block costs the thread that issues the products about 0.37 us (0.49 us for a gate/up pair), more
+// kernel: a k-block costs the thread that issues the products about 0.37 us (0.49 us for a gate/up pair; with two
+// issuing threads half of that, which is also what the tensor pipe itself then needs for narrow products: about 85
+// cycles each whatever their width, since each fetches its 4 KB slab of weight rows from shared memory), more
 // when shared memory (128 B per cycle for the incoming stage plus the operand reads of every product) or the
 // block's intake (about 150 GB/s; the whole chip about 25 TB/s out of L2, weights about 6 TB/s out of HBM) is slower; the first operands arrive about 1 us after they were asked for; the epilogue
 // costs about 0.5 us per 32 tokens (only the last tile's is exposed); and a k-split over a cluster adds
